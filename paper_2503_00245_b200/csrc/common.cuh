@@ -1,0 +1,215 @@
+// Shared host/device helpers for the MoE layer kernels (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/cosmoe.h"
+
+namespace cosmoe {
+
+// ------------------------------------------------------------------ host side
+extern thread_local int g_last_cuda_error;
+
+#define MOE_CUDA_TRY(expr)                   \
+  do {                                       \
+    cudaError_t _e = (expr);                 \
+    if (_e != cudaSuccess) {                 \
+      ::cosmoe::g_last_cuda_error = (int)_e; \
+      (void)cudaGetLastError();              \
+      return MOE_ERR_CUDA;                   \
+    }                                        \
+  } while (0)
+
+// Device-resident state of a ctx: status word written by kernels, grid barrier.
+struct DeviceState {
+  unsigned int status;     // 0 ok, else moe_status
+  unsigned int detail;     // where it happened (kernel-specific code)
+  unsigned int bar_count;  // arrivals at the current grid barrier
+  unsigned int bar_gen;    // generation, bumped by the last arriver
+};
+
+}  // namespace cosmoe
+
+struct moe_ctx {
+  moe_config cfg;
+  int device;
+  int sm_count;
+  int max_smem_optin;
+  cosmoe::DeviceState* d_state;  // device
+  cosmoe::DeviceState* h_state;  // pinned host mirror for moe_check
+  unsigned long long launches;
+};
+
+namespace cosmoe {
+
+// Offsets (bytes) of the pieces of the caller's scratch buffer.
+struct WsLayout {
+  size_t topk_idx, topk_w, offsets, perm, inv;  // routing products when the caller does not ask for them
+  size_t vec_a, vec_b, vec_c;                   // fp32 inter-phase vectors of the streaming path
+  size_t xperm, hidden, mid_a, mid_b;           // bf16 operands of the tensor path
+  size_t out_slots;                             // fp32 [T*k][d]
+  size_t total;
+};
+WsLayout ws_layout(const moe_config& c, int T);
+
+int validate_config(const moe_config* c);
+
+// launchers implemented in the other translation units
+int launch_route(moe_ctx* ctx, const void* x, int T, const moe_weights* w, int32_t* idx, float* wt, float* probs,
+                 cudaStream_t s);
+int launch_permute(moe_ctx* ctx, const int32_t* idx, int T, int32_t* offsets, int32_t* perm, int32_t* inv,
+                   cudaStream_t s);
+int launch_combine(moe_ctx* ctx, const float* out_slots, const float* wt, const int32_t* inv, int T, void* y,
+                   cudaStream_t s);
+int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_slots, void* xperm, cudaStream_t s);
+
+// Streaming (decode) path.  mode 0: whole layer from topk (writes y); mode 1: FFN per slot from
+// expert_offsets/perm (writes out_slots).
+int launch_stream_ffn(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, const int32_t* topk_idx,
+                      const float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
+                      char* ws, const WsLayout& L, cudaStream_t s);
+// Tensor-core (prefill) path: out_slots from x gathered by perm.
+int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, const int32_t* offsets,
+                      const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, cudaStream_t s);
+
+// ------------------------------------------------------------------ device side
+#ifdef __CUDACC__
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Longest any device-side wait may last before the kernel gives up and flags MOE_ERR_TIMEOUT.
+constexpr uint64_t kWaitBudgetNs = 2000000000ull;
+
+__device__ __forceinline__ void flag_error(DeviceState* st, unsigned code, unsigned detail) {
+  if (atomicCAS(&st->status, 0u, code) == 0u) st->detail = detail;
+}
+
+// ---- mbarrier -----------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the budget ran out (the barrier never completed its phase).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_timer_ns() - t0 > kWaitBudgetNs) return false;
+  }
+}
+
+// ---- bulk asynchronous copy global -> shared (TMA, no tensor map) ---------------
+// src and dst 16-byte aligned, bytes a multiple of 16.  Completion is counted on `bar`.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst_smem)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// ---- acquire / release on global words -------------------------------------------
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned atom_add_acq_rel(unsigned* p, unsigned v) {
+  unsigned old;
+  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+
+// Barrier over all CTAs of a co-resident (cooperative) grid.  Thread 0 of each CTA arrives; the
+// wait is bounded.  Returns false (for the whole CTA) when the budget ran out.
+__device__ __forceinline__ bool grid_barrier(DeviceState* st, unsigned n_ctas, int* smem_flag) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int ok = 1;
+    const unsigned gen = ld_acquire(&st->bar_gen);
+    __threadfence();
+    const unsigned old = atom_add_acq_rel(&st->bar_count, 1u);
+    if (old == n_ctas - 1u) {
+      st->bar_count = 0u;
+      __threadfence();
+      st_release(&st->bar_gen, gen + 1u);
+    } else {
+      const uint64_t t0 = global_timer_ns();
+      while (ld_acquire(&st->bar_gen) == gen) {
+        if (global_timer_ns() - t0 > kWaitBudgetNs) {
+          ok = 0;
+          break;
+        }
+      }
+    }
+    __threadfence();
+    *smem_flag = ok;
+  }
+  __syncthreads();
+  return *smem_flag != 0;
+}
+
+// ---- bf16 helpers ---------------------------------------------------------------------
+// 8 bf16 packed in a uint4 -> 8 floats (exact).
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  f[0] = __uint_as_float(v.x << 16);
+  f[1] = __uint_as_float(v.x & 0xffff0000u);
+  f[2] = __uint_as_float(v.y << 16);
+  f[3] = __uint_as_float(v.y & 0xffff0000u);
+  f[4] = __uint_as_float(v.z << 16);
+  f[5] = __uint_as_float(v.z & 0xffff0000u);
+  f[6] = __uint_as_float(v.w << 16);
+  f[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+__device__ __forceinline__ float bf16_to_float(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
+
+#endif  // __CUDACC__
+}  // namespace cosmoe
