@@ -1,0 +1,338 @@
+// Router (logits + softmax + top-k + gate weights), token->expert grouping, row gather,
+// gate-weighted combine and the one-off weight packing kernels.
+#include "common.cuh"
+
+namespace cosmoe {
+
+// ------------------------------------------------------------------------------------ router
+// One warp per token.  Lanes split the d axis; every lane keeps E partial logits, a shuffle
+// tree finishes them, lane 0 does the E-wide softmax / top-k serially (E <= 64).
+// Selection runs on the logits: softmax is monotonic, so top_k(W) = top_k(R) (Eq. 2, Eq. 3), and
+// the logits carry more bits than the fp32 probabilities.  Ties go to the lower expert index.
+template <typename XT>
+__device__ __forceinline__ void load_x8(const XT* p, float* f);
+template <>
+__device__ __forceinline__ void load_x8<float>(const float* p, float* f) {
+  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  f[0] = a.x, f[1] = a.y, f[2] = a.z, f[3] = a.w, f[4] = b.x, f[5] = b.y, f[6] = b.z, f[7] = b.w;
+}
+template <>
+__device__ __forceinline__ void load_x8<__nv_bfloat16>(const __nv_bfloat16* p, float* f) {
+  unpack8(*reinterpret_cast<const uint4*>(p), f);
+}
+
+constexpr int kRouteWarps = 8;
+
+template <typename XT, int EMAX>
+__global__ void __launch_bounds__(kRouteWarps * 32)
+    route_kernel(const XT* __restrict__ x, const uint16_t* __restrict__ w_router, const float* __restrict__ bias, int T,
+                 int d, int E, int k, int renorm, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
+                 float* __restrict__ probs) {
+  __shared__ float s_logit[kRouteWarps][EMAX];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int t = blockIdx.x * kRouteWarps + wib;
+  if (t >= T) return;
+  float acc[EMAX];
+#pragma unroll
+  for (int e = 0; e < EMAX; ++e) acc[e] = 0.f;
+  const XT* xr = x + (size_t)t * d;
+  const bool vec = (E % 8) == 0;
+  for (int c = lane; c < d / 8; c += 32) {
+    float xv[8];
+    load_x8<XT>(xr + c * 8, xv);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint16_t* wr = w_router + (size_t)(c * 8 + i) * E;
+      if (vec) {
+#pragma unroll
+        for (int e8 = 0; e8 < EMAX / 8; ++e8) {
+          if (e8 * 8 < E) {
+            float wv[8];
+            unpack8(__ldg(reinterpret_cast<const uint4*>(wr) + e8), wv);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[e8 * 8 + j] = fmaf(xv[i], wv[j], acc[e8 * 8 + j]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < EMAX; ++e)
+          if (e < E) acc[e] = fmaf(xv[i], bf16_to_float(__ldg(wr + e)), acc[e]);
+      }
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < EMAX; ++e)
+    if (e < E) acc[e] = warp_sum(acc[e]);
+  if (lane == 0) {
+#pragma unroll
+    for (int e = 0; e < EMAX; ++e)
+      if (e < E) s_logit[wib][e] = acc[e] + (bias ? bias[e] : 0.f);
+    float* lg = s_logit[wib];
+    float m = lg[0];
+    for (int e = 1; e < E; ++e) m = fmaxf(m, lg[e]);
+    float sum = 0.f;
+    for (int e = 0; e < E; ++e) sum += expf(lg[e] - m);
+    const float inv_sum = 1.0f / sum;
+    if (probs)
+      for (int e = 0; e < E; ++e) probs[(size_t)t * E + e] = expf(lg[e] - m) * inv_sum;
+    unsigned long long taken = 0ull;
+    float wsel[MOE_MAX_TOPK];
+    float wtot = 0.f;
+    for (int j = 0; j < k; ++j) {
+      int best = -1;
+      float bv = 0.f;
+      for (int e = 0; e < E; ++e) {
+        if ((taken >> e) & 1ull) continue;
+        if (best < 0 || lg[e] > bv) best = e, bv = lg[e];
+      }
+      taken |= 1ull << best;
+      topk_idx[(size_t)t * k + j] = best;
+      wsel[j] = expf(bv - m) * inv_sum;
+      wtot += wsel[j];
+    }
+    const float scale = renorm ? 1.0f / wtot : 1.0f;
+    for (int j = 0; j < k; ++j) topk_w[(size_t)t * k + j] = wsel[j] * scale;
+  }
+}
+
+template <typename XT>
+static int launch_route_t(moe_ctx* ctx, const void* x, int T, const moe_weights* w, int32_t* idx, float* wt,
+                          float* probs, cudaStream_t s) {
+  const moe_config& c = ctx->cfg;
+  const dim3 grid((T + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
+  const XT* xp = (const XT*)x;
+  const uint16_t* wr = (const uint16_t*)w->w_router;
+#define ROUTE_CASE(EM)                                                                                               \
+  route_kernel<XT, EM><<<grid, block, 0, s>>>(xp, wr, w->b_router, T, c.d_model, c.n_experts, c.top_k, c.renorm, idx, \
+                                              wt, probs)
+  if (c.n_experts <= 8)
+    ROUTE_CASE(8);
+  else if (c.n_experts <= 16)
+    ROUTE_CASE(16);
+  else if (c.n_experts <= 32)
+    ROUTE_CASE(32);
+  else
+    ROUTE_CASE(64);
+#undef ROUTE_CASE
+  MOE_CUDA_TRY(cudaGetLastError());
+  ctx->launches++;
+  return MOE_OK;
+}
+
+int launch_route(moe_ctx* ctx, const void* x, int T, const moe_weights* w, int32_t* idx, float* wt, float* probs,
+                 cudaStream_t s) {
+  if (ctx->cfg.x_dtype == MOE_F32) return launch_route_t<float>(ctx, x, T, w, idx, wt, probs, s);
+  return launch_route_t<__nv_bfloat16>(ctx, x, T, w, idx, wt, probs, s);
+}
+
+// ------------------------------------------------------------------------------------ grouping
+// One CTA: histogram of the T*k pairs by expert, exclusive scan, then a stable scatter that walks
+// the pairs in order, 1024 at a time (rank inside a warp by match_any, across warps by a scan).
+constexpr int kPermThreads = 1024;
+
+__global__ void __launch_bounds__(kPermThreads)
+    permute_kernel(const int32_t* __restrict__ topk_idx, int n, int E, int32_t* __restrict__ offsets,
+                   int32_t* __restrict__ perm, int32_t* __restrict__ inv, DeviceState* st) {
+  __shared__ int s_base[MOE_MAX_EXPERTS];
+  __shared__ int s_wc[kPermThreads / 32][MOE_MAX_EXPERTS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid < MOE_MAX_EXPERTS) s_base[tid] = 0;
+  __syncthreads();
+  for (int p = tid; p < n; p += kPermThreads) {
+    const int e = topk_idx[p];
+    if (e < 0 || e >= E)
+      flag_error(st, MOE_ERR_STATE, 0x100u);
+    else
+      atomicAdd(&s_base[e], 1);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int e = 0; e < E; ++e) {
+      const int c = s_base[e];
+      offsets[e] = run;
+      s_base[e] = run;
+      run += c;
+    }
+    offsets[E] = run;
+  }
+  __syncthreads();
+  for (int p0 = 0; p0 < n; p0 += kPermThreads) {
+    for (int i = tid; i < (kPermThreads / 32) * MOE_MAX_EXPERTS; i += kPermThreads) (&s_wc[0][0])[i] = 0;
+    __syncthreads();
+    const int p = p0 + tid;
+    int e = -1;
+    if (p < n) {
+      e = topk_idx[p];
+      if (e < 0 || e >= E) e = -1;
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    if (e >= 0 && rank == 0) s_wc[warp][e] = __popc(peers);
+    __syncthreads();
+    if (tid < E) {
+      int run = s_base[tid];
+      for (int w = 0; w < kPermThreads / 32; ++w) {
+        const int c = s_wc[w][tid];
+        s_wc[w][tid] = run;
+        run += c;
+      }
+      s_base[tid] = run;
+    }
+    __syncthreads();
+    if (e >= 0) {
+      const int slot = s_wc[warp][e] + rank;
+      perm[slot] = p;
+      inv[p] = slot;
+    }
+    __syncthreads();
+  }
+}
+
+int launch_permute(moe_ctx* ctx, const int32_t* idx, int T, int32_t* offsets, int32_t* perm, int32_t* inv,
+                   cudaStream_t s) {
+  const moe_config& c = ctx->cfg;
+  permute_kernel<<<1, kPermThreads, 0, s>>>(idx, T * c.top_k, c.n_experts, offsets, perm, inv, ctx->d_state);
+  MOE_CUDA_TRY(cudaGetLastError());
+  ctx->launches++;
+  return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------ gather
+// xperm[s][:] = bf16(x[perm[s] / k][:])  (operand rows of the tensor-core path, grouped by expert)
+template <typename XT>
+__global__ void gather_rows_kernel(const XT* __restrict__ x, const int32_t* __restrict__ perm, int n_slots, int k,
+                                   int d, uint4* __restrict__ out) {
+  const int chunks = d / 8;
+  const long long total = (long long)n_slots * chunks;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int s = (int)(i / chunks), c = (int)(i % chunks);
+    const int t = perm[s] / k;
+    float f[8];
+    load_x8<XT>(x + (size_t)t * d + c * 8, f);
+    uint4 o;
+    o.x = pack_bf16x2(f[0], f[1]), o.y = pack_bf16x2(f[2], f[3]);
+    o.z = pack_bf16x2(f[4], f[5]), o.w = pack_bf16x2(f[6], f[7]);
+    out[i] = o;
+  }
+}
+
+int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_slots, void* xperm, cudaStream_t s) {
+  const moe_config& c = ctx->cfg;
+  const long long total = (long long)n_slots * (c.d_model / 8);
+  const int block = 256;
+  const int grid = (int)((total + block - 1) / block < 148 * 16 ? (total + block - 1) / block : 148 * 16);
+  if (c.x_dtype == MOE_F32)
+    gather_rows_kernel<float><<<grid, block, 0, s>>>((const float*)x, perm, n_slots, c.top_k, c.d_model, (uint4*)xperm);
+  else
+    gather_rows_kernel<__nv_bfloat16>
+        <<<grid, block, 0, s>>>((const __nv_bfloat16*)x, perm, n_slots, c.top_k, c.d_model, (uint4*)xperm);
+  MOE_CUDA_TRY(cudaGetLastError());
+  ctx->launches++;
+  return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------ combine
+// y[t][c] = sum_j w[t][j] * out_slots[inv[t*k+j]][c], j ascending, fp32, one rounding to the output type.
+template <typename YT>
+__global__ void combine_kernel(const float* __restrict__ out_slots, const float* __restrict__ wt,
+                               const int32_t* __restrict__ inv, int T, int k, int d, YT* __restrict__ y) {
+  const int quads = d / 4;
+  const long long total = (long long)T * quads;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int t = (int)(i / quads), q = (int)(i % quads);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < k; ++j) {
+      const float w = wt[(size_t)t * k + j];
+      const float4 o = *reinterpret_cast<const float4*>(out_slots + (size_t)inv[(size_t)t * k + j] * d + q * 4);
+      acc.x = fmaf(w, o.x, acc.x), acc.y = fmaf(w, o.y, acc.y), acc.z = fmaf(w, o.z, acc.z), acc.w = fmaf(w, o.w, acc.w);
+    }
+    if constexpr (sizeof(YT) == 4) {
+      *reinterpret_cast<float4*>(y + (size_t)t * d + q * 4) = acc;
+    } else {
+      uint2 o;
+      o.x = pack_bf16x2(acc.x, acc.y), o.y = pack_bf16x2(acc.z, acc.w);
+      *reinterpret_cast<uint2*>(y + (size_t)t * d + q * 4) = o;
+    }
+  }
+}
+
+int launch_combine(moe_ctx* ctx, const float* out_slots, const float* wt, const int32_t* inv, int T, void* y,
+                   cudaStream_t s) {
+  const moe_config& c = ctx->cfg;
+  const long long total = (long long)T * (c.d_model / 4);
+  const int block = 256;
+  const int grid = (int)((total + block - 1) / block < 148 * 16 ? (total + block - 1) / block : 148 * 16);
+  if (c.x_dtype == MOE_F32)
+    combine_kernel<float><<<grid, block, 0, s>>>(out_slots, wt, inv, T, c.top_k, c.d_model, (float*)y);
+  else
+    combine_kernel<__nv_bfloat16><<<grid, block, 0, s>>>(out_slots, wt, inv, T, c.top_k, c.d_model, (__nv_bfloat16*)y);
+  MOE_CUDA_TRY(cudaGetLastError());
+  ctx->launches++;
+  return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------ packing
+// in [B][R][C] -> out[b][c][sub][r] with nsub interleaved row kinds: a tiled transpose.
+__global__ void pack_transpose_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, int R, int C,
+                                      int nsub, int sub) {
+  __shared__ uint16_t tile[32][33];
+  const int b = blockIdx.z;
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const uint16_t* src = in + (size_t)b * R * C;
+  uint16_t* dst = out + (size_t)b * C * nsub * R;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int r = r0 + i, c = c0 + threadIdx.x;
+    if (r < R && c < C) tile[i][threadIdx.x] = src[(size_t)r * C + c];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int c = c0 + i, r = r0 + threadIdx.x;
+    if (r < R && c < C) dst[((size_t)c * nsub + sub) * R + r] = tile[threadIdx.x][i];
+  }
+}
+
+static int pack_one(const void* in, void* out, int B, int R, int C, int nsub, int sub, cudaStream_t s) {
+  const dim3 grid((C + 31) / 32, (R + 31) / 32, B), block(32, 8);
+  if (grid.y > 65535u || grid.z > 65535u) return MOE_ERR_UNSUPPORTED;
+  pack_transpose_kernel<<<grid, block, 0, s>>>((const uint16_t*)in, (uint16_t*)out, R, C, nsub, sub);
+  MOE_CUDA_TRY(cudaGetLastError());
+  return MOE_OK;
+}
+
+}  // namespace cosmoe
+
+using namespace cosmoe;
+
+extern "C" {
+
+int moe_pack_dense(int32_t d, int32_t f, int32_t n_experts, const void* w_gate, const void* w_up, const void* w_down,
+                   void* gate_up_out, void* down_t_out, void* stream) {
+  if (d <= 0 || f <= 0 || n_experts <= 0 || !w_gate || !w_up || !w_down || !gate_up_out || !down_t_out)
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc = pack_one(w_gate, gate_up_out, n_experts, d, f, 2, 0, s);
+  if (rc == MOE_OK) rc = pack_one(w_up, gate_up_out, n_experts, d, f, 2, 1, s);
+  if (rc == MOE_OK) rc = pack_one(w_down, down_t_out, n_experts, f, d, 1, 0, s);
+  return rc;
+}
+
+int moe_pack_wd(int32_t d, int32_t f, int32_t r, int32_t n_experts, const void* gL, const void* gR, const void* uL,
+                const void* uR, const void* dL, const void* dR, void* wd_a, void* wd_b, void* wd_c, void* wd_d,
+                void* stream) {
+  if (d <= 0 || f <= 0 || r <= 0 || n_experts <= 0 || !gL || !gR || !uL || !uR || !dL || !dR || !wd_a || !wd_b ||
+      !wd_c || !wd_d)
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc = pack_one(gL, wd_a, n_experts, d, r, 2, 0, s);
+  if (rc == MOE_OK) rc = pack_one(uL, wd_a, n_experts, d, r, 2, 1, s);
+  if (rc == MOE_OK) rc = pack_one(gR, wd_b, n_experts, r, f, 2, 0, s);
+  if (rc == MOE_OK) rc = pack_one(uR, wd_b, n_experts, r, f, 2, 1, s);
+  if (rc == MOE_OK) rc = pack_one(dL, wd_c, n_experts, f, r, 1, 0, s);
+  if (rc == MOE_OK) rc = pack_one(dR, wd_d, n_experts, r, d, 1, 0, s);
+  return rc;
+}
+
+}  // extern "C"

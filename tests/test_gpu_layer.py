@@ -1,0 +1,91 @@
+"""GPU parity of moe_layer_forward against the CPU checker: the paper-shaped configurations and
+the degenerate cases, streaming (decode) and tensor-core (prefill) paths."""
+import numpy as np
+import pytest
+import torch
+
+from synth import workloads as W
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+STREAM, TENSOR = 1, 2
+
+
+def shape(d, f, E=8, k=2, r=0, xd="bf16", bias="none", cfg_id=8):
+    return W.LayerShape("t", cfg_id, d, f, n_experts=E, top_k=k, wd_rank=r, x_dtype=xd, bias=bias)
+
+
+@pytest.mark.parametrize("sh,T,path", [
+    (W.TINY, 16, STREAM),
+    (W.TINY, 16, TENSOR),
+    (W.WEARABLE, 1, 0),
+    (W.WEARABLE, 8, 0),
+    (W.WEARABLE, 512, 0),
+    (W.PHONE, 1, 0),
+    (W.PHONE_WD128, 1, 0),
+    (W.PHONE_WD1024, 1, 0),
+    (W.PHONE_OFFLOAD, 1, 0),                        # E = 16, Zipf bias
+    (shape(1440, 3840), 1, 0),                      # the paper's own phone-sized layer (Table 1 widths)
+    (shape(432, 1280), 3, 0),                       # the paper's wearable-sized layer
+    (shape(136, 200, E=6, k=3), 5, STREAM),
+    (shape(256, 512, k=1), 4, STREAM),
+    (shape(256, 512, k=8), 2, STREAM),
+    (shape(256, 512, r=64), 16, STREAM),
+    (shape(256, 512, r=64, xd="f32"), 7, STREAM),
+])
+def test_layer_forward_matches_checker(sh, T, path):
+    lay, t, host = U.build(sh, T, path=path)
+    rel, _, _ = U.check_layer(lay, t, host, sh.top_k)
+    assert rel <= U.Y_TOL
+
+
+def test_all_tokens_to_one_expert_stream():
+    """Bias forces expert 5 into every token's set: one expert serves 16 tokens (two passes of 8),
+    most experts get nothing."""
+    sh = shape(256, 512)
+    t = W.make_layer(sh, 16, device="cuda")
+    b = torch.zeros(8, device="cuda")
+    b[5] = 50.0
+    t["b_router"] = b
+    lay, t, host = U.build(sh, 16, path=STREAM, tensors=t)
+    rel, ora, _ = U.check_layer(lay, t, host, 2)
+    assert ora["counts"][5] == 16 and (ora["counts"] == 0).sum() >= 1
+
+
+def test_layer_equals_composition_of_steps():
+    sh = W.WEARABLE
+    lay, t, host = U.build(sh, 8)
+    y = lay.forward(t["x"])
+    idx, w, _ = lay.route(t["x"])
+    offsets, perm, inv = lay.permute(idx)
+    out = lay.expert_ffn(t["x"], offsets, perm)
+    y2 = lay.combine(out, w, inv)
+    torch.cuda.synchronize()
+    assert lay.check() == 0
+    a, b = y.float(), y2.float()
+    assert torch.max(torch.abs(a - b)) <= 2.0 ** -7 * torch.sqrt(torch.mean(b * b))   # one bf16 ulp of slack
+
+
+def test_repeat_calls_are_bitwise_identical():
+    lay, t, _ = U.build(W.WEARABLE, 8)
+    y1 = lay.forward(t["x"]).clone()
+    y2 = lay.forward(t["x"]).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+
+
+def test_argument_errors_are_reported_not_run():
+    from paper_2503_00245_b200 import binding as B
+    lay, t, _ = U.build(W.TINY, 16)
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    y = torch.empty_like(t["x"])
+    with pytest.raises(B.MoeError) as e:
+        B.moe_layer_forward(lay.ctx, t["x"], 16, lay.weights, y, ws=small)
+    assert e.value.status == 3
+    lay2, t2, _ = U.build(W.TINY, 32, path=STREAM, max_tokens=32)
+    with pytest.raises(B.MoeError) as e:
+        lay2.forward(t2["x"])
+    assert e.value.status == 2                      # streaming path is limited to 16 tokens
+    B.moe_layer_forward(lay.ctx, t["x"], 0, lay.weights, y, ws=lay.ws)   # T = 0: no-op
+    assert lay.check() == 0
