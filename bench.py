@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE feed-forward layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--all] [--impl reference]
+
+One step = one forward pass of the whole layer (router, top-k gating, grouping, expert FFN,
+gate-weighted combine) over one batch of seeded synthetic input.  The default workload is the
+wearables-scale layer at batch-1 decode; steps walk a ring of distinct layers whose touched
+weights exceed the L2 several times over, so every step reads its experts from HBM.
+Prints ONE JSON line (see the keys below).  N > 1: independent replicas, one per GPU, no collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from synth import workloads as W  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+
+WORKLOADS = {
+    # name: (shape, T, kind)
+    "wearable-decode-T1": (W.WEARABLE, 1, "decode"),
+    "wearable-decode-T8": (W.WEARABLE, 8, "decode"),
+    "wearable-prefill-T512": (W.WEARABLE, 512, "prefill"),
+    "phone-decode-T1": (W.PHONE, 1, "decode"),
+    "phone-prefill-T2048": (W.PHONE, 2048, "prefill"),
+    "phone-wd128-decode-T1": (W.PHONE_WD128, 1, "decode"),
+    "phone-wd1024-decode-T1": (W.PHONE_WD1024, 1, "decode"),
+    "phone-wd128-prefill-T2048": (W.PHONE_WD128, 2048, "prefill"),
+    "phone-wd1024-prefill-T2048": (W.PHONE_WD1024, 2048, "prefill"),
+    "tiny-T16": (W.TINY, 16, "decode"),
+}
+DEFAULT = "wearable-decode-T1"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        m = json.load(open(p))
+        return {"hbm_gbs": m["hbm_gbs"], "tflops": m["bf16_tflops"], "tflops_sustained": m["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def algorithmic_bytes(shape: W.LayerShape, n_active_experts: float, T: int) -> float:
+    """Bytes one layer forward must move: the selected experts' weights once, the router, x and y."""
+    d, E = shape.d_model, shape.n_experts
+    return n_active_experts * W.expert_bytes(shape) + 2 * d * E + 2 * 2 * T * d
+
+
+def flops(shape: W.LayerShape, T: int) -> float:
+    per = 6 * shape.wd_rank * (shape.d_model + shape.d_ff) if shape.wd_rank else 6 * shape.d_model * shape.d_ff
+    return float(T) * shape.top_k * per + 2.0 * T * shape.d_model * shape.n_experts
+
+
+def build_ring(shape, T, device, min_touched_bytes, ring_override=0):
+    """Distinct layers (weights + inputs) so that consecutive steps never find their experts in L2."""
+    import paper_2503_00245_b200 as P
+    touched = min(shape.n_experts, T * shape.top_k) * W.expert_bytes(shape)
+    n_layers = max(2, -(-min_touched_bytes // touched))
+    n_layers = min(n_layers, 64)
+    if ring_override:
+        n_layers = ring_override
+    kw = dict(d_model=shape.d_model, d_ff=shape.d_ff, n_experts=shape.n_experts, top_k=shape.top_k)
+    ring = []
+    for l in range(n_layers):
+        t = W.make_layer(shape, T, device=device, layer=l)
+        lay = P.MoELayer.from_math_layout(kw, t, x_dtype=t["x"].dtype, max_tokens=T)
+        x = t["x"]
+        ring.append({"layer": lay, "x": x, "y": torch.empty_like(x),
+                     "idx": torch.empty((T, shape.top_k), dtype=torch.int32, device=device),
+                     "w": torch.empty((T, shape.top_k), dtype=torch.float32, device=device)})
+        del t
+    torch.cuda.synchronize()
+    return ring
+
+
+def run_ring(ring, steps, start=0):
+    n = len(ring)
+    for i in range(steps):
+        r = ring[(start + i) % n]
+        r["layer"].forward(r["x"], y=r["y"], topk_idx=r["idx"], topk_w=r["w"])
+
+
+def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use_graph=True):
+    shape, T, kind = WORKLOADS[name]
+    pk = peaks()
+    ring = build_ring(shape, T, device, 4 * L2_BYTES, ring_override)
+    n = len(ring)
+    stream = torch.cuda.current_stream()
+    launches0 = sum(_launches(r) for r in ring)
+    run_ring(ring, max(warmup, 3))
+    torch.cuda.synchronize()
+    for r in ring:
+        assert r["layer"].check() == 0, "a kernel flagged an error during warm-up"
+    launches_per_step = (sum(_launches(r) for r in ring) - launches0) / max(warmup, 3)
+
+    # CUDA graph of one trip around the ring (decode steps are launch-bound otherwise)
+    graph = None
+    mode = "stream"
+    if kind == "decode" and use_graph:
+        try:
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                run_ring(ring, n)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=side):
+                    run_ring(ring, n)
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            graph, mode = g, "cuda_graph"
+        except Exception as e:  # noqa: BLE001
+            sys.stderr.write(f"[bench] CUDA graph capture unavailable ({e}); timing plain launches\n")
+            torch.cuda.synchronize()
+            graph = None
+    trips = max(1, steps // n) if graph is not None else None
+    steps_eff = trips * n if graph is not None else steps
+
+    def timed_once():
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        e0.record()
+        if graph is not None:
+            for _ in range(trips):
+                graph.replay()
+        else:
+            run_ring(ring, steps_eff)
+        e1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        return e0.elapsed_time(e1)
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    ms = timed_once()
+    # keep the GPU busy long enough for at least a few clock samples
+    extra_ms, reps = 0.0, 0
+    while sampler and (extra_ms + ms) < 400.0 and reps < 50:
+        extra_ms += timed_once()
+        reps += 1
+    clocks = sampler.stop() if sampler else None
+    if reps:
+        ms = (ms + extra_ms) / (reps + 1)
+    for r in ring:
+        assert r["layer"].check() == 0, "a kernel flagged an error during the timed region"
+
+    # distinct experts actually read per step (exact, from the routing the kernels produced)
+    act = sum(len(set(r["idx"].flatten().tolist())) for r in ring) / n
+    res = {"name": name, "shape": shape, "T": T, "kind": kind, "ms_total": ms, "steps": steps_eff,
+           "ms_per_step": ms / steps_eff, "launch_mode": mode, "ring_layers": n, "active_experts_per_step": act,
+           "launches_per_step": launches_per_step, "clocks": clocks, "peaks": pk, "ring": ring}
+    return res
+
+
+def _launches(r):
+    from paper_2503_00245_b200 import binding as B
+    return B.moe_launch_count(r["layer"].ctx)
+
+
+def roofline(res):
+    shape, T, pk = res["shape"], res["T"], res["peaks"]
+    sec = res["ms_per_step"] * 1e-3
+    if res["kind"] == "decode":
+        b = algorithmic_bytes(shape, res["active_experts_per_step"], T)
+        ach = b / sec / 1e9
+        return {"bound": "hbm", "achieved": round(ach, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": round(ach / pk["hbm_gbs"], 4), "traffic": None, "peak_source": pk["source"],
+                "bytes_per_launch": int(b), "kernel": "stream_ffn_kernel",
+                "note": "duration = whole step (router + expert kernel) / 1"}
+    fl = flops(shape, T)
+    t_tc = fl / (pk["tflops_sustained"] * 1e12)
+    t_hbm = algorithmic_bytes(shape, shape.n_experts, T) / (pk["hbm_gbs"] * 1e9)
+    if t_hbm > t_tc:
+        b = algorithmic_bytes(shape, shape.n_experts, T)
+        ach = b / sec / 1e9
+        return {"bound": "hbm", "achieved": round(ach, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": round(ach / pk["hbm_gbs"], 4), "traffic": None, "peak_source": pk["source"],
+                "tensor_tflops": round(fl / sec / 1e12, 1)}
+    ach = fl / sec / 1e12
+    return {"bound": "tensor", "achieved": round(ach, 1), "peak": pk["tflops_sustained"], "unit": "TFLOP/s",
+            "frac": round(ach / pk["tflops_sustained"], 4), "traffic": None, "peak_source": pk["source"],
+            "peak_kind": "sustained bf16 (kernel timed inside a long step)"}
+
+
+def e2e_measure(res, steps):
+    """Same metric through the public call with HOST buffers: pinned x -> device, layer, y -> host, per step."""
+    ring = res["ring"]
+    T, shape = res["T"], res["shape"]
+    n = len(ring)
+    hx = [r["x"].cpu().pin_memory() for r in ring]
+    hy = [torch.empty_like(h).pin_memory() for h in hx]
+    steps = min(steps, 2000)
+    for i in range(min(8, steps)):
+        r = ring[i % n]
+        r["x"].copy_(hx[i % n], non_blocking=True)
+        r["layer"].forward(r["x"], y=r["y"])
+        hy[i % n].copy_(r["y"], non_blocking=True)
+        torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(steps):
+        r = ring[i % n]
+        r["x"].copy_(hx[i % n], non_blocking=True)
+        r["layer"].forward(r["x"], y=r["y"])
+        hy[i % n].copy_(r["y"], non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller reads y before the next token
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    nbytes = hx[0].numel() * hx[0].element_size()
+    return ms, nbytes, nbytes
+
+
+def metric_of(res, ms_per_step, world=1):
+    T = res["T"]
+    if res["kind"] == "decode":
+        return "moe_layer_us_per_token_decode", ms_per_step * 1e3 / (T * world), "us/token", False
+    return "moe_layer_prefill_tokens_per_s", T * world / (ms_per_step * 1e-3), "tokens/s", True
+
+
+def cpu_baseline(name, budget_s=12.0):
+    """The CPU checker as it stands, timed on this machine's host cores on the same workload."""
+    import numpy as np
+    from threadpoolctl import threadpool_info
+    from oracle import moe_oracle as O
+    shape, T, kind = WORKLOADS[name]
+    t = W.make_layer(shape, T, device="cpu", layer=0)
+    h = {k: W.to_host_bits(v) for k, v in t.items()}
+    ex = {k: v for k, v in h.items() if k not in ("x", "w_router", "b_router")}
+    O.layer_forward(h["x"], h["w_router"], h["b_router"], ex, shape.top_k)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        O.layer_forward(h["x"], h["w_router"], h["b_router"], ex, shape.top_k)
+        n += 1
+        el = time.perf_counter() - t0
+        if el > budget_s or n >= 2000:
+            break
+    per = el / n
+    threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    if kind == "decode":
+        val, unit = per * 1e6 / T, "us/token"
+    else:
+        val, unit = T / per, "tokens/s"
+    return {"value": round(val, 3), "unit": unit, "cores": int(threads), "kind": "oracle",
+            "sample": f"{n} forward passes of layer 0 of the ring ({el:.1f} s of CPU time), numpy fp64"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4096)
+    ap.add_argument("--warmup", type=int, default=64)
+    ap.add_argument("--workload", default=DEFAULT, choices=sorted(WORKLOADS))
+    ap.add_argument("--all", action="store_true", help="also time the other workloads (reported under 'others')")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ring", type=int, default=0, help="override the number of distinct layers in the ring")
+    ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
+    a = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    a.warmup = max(a.warmup, 3)
+
+    if a.impl == "reference":
+        if rank != 0:
+            return 0
+        shape, T, kind = WORKLOADS[a.workload]
+        cb = cpu_baseline(a.workload, budget_s=min(60.0, 2.0 * max(1, a.steps // 512)))
+        line = {"impl": "reference", "metric": metric_of({"T": T, "kind": kind}, 1.0)[0], "value": cb["value"],
+                "unit": cb["unit"], "n_gpus": 0, "steps": a.steps, "warmup": a.warmup,
+                "ms_per_step": cb["value"] * T / 1e3 if kind == "decode" else T / cb["value"] * 1e3,
+                "higher_is_better": kind != "decode", "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic", "config": {"workload": a.workload, "shape": W.describe(shape), "T": T},
+                "cpu_baseline": cb,
+                "e2e": {"value": cb["value"], "unit": cb["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return 0
+
+    if not torch.cuda.is_available():
+        sys.stderr.write("bench.py: no CUDA device; the layer has no CPU fallback\n")
+        return 2
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    from paper_2503_00245_b200 import build as _b
+    if rank == 0:
+        _b.build()
+    if world > 1:
+        torch.distributed.barrier()
+
+    res = time_workload(a.workload, a.steps, a.warmup, device, rank, world, a.ring, not a.no_graph)
+    ms_tot = torch.tensor([res["ms_total"]], device=device, dtype=torch.float64)
+    if world > 1:
+        torch.distributed.all_reduce(ms_tot, op=torch.distributed.ReduceOp.MAX)
+    ms_per_step = float(ms_tot.item()) / res["steps"]
+    metric, value, unit, hib = metric_of(res, ms_per_step, world)
+    e2e_ms, h2d, d2h = e2e_measure(res, a.steps)
+    e2e_t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
+    if world > 1:
+        torch.distributed.all_reduce(e2e_t, op=torch.distributed.ReduceOp.MAX)
+    _, e2e_val, _, _ = metric_of(res, float(e2e_t.item()), world)
+
+    others = []
+    if a.all and rank == 0 and world == 1:
+        del res["ring"]
+        torch.cuda.empty_cache()
+        for name in WORKLOADS:
+            if name == a.workload:
+                continue
+            try:
+                r = time_workload(name, a.steps, a.warmup, device, rank, 1)
+            except Exception as e:  # noqa: BLE001
+                others.append({"workload": name, "error": str(e)[:200]})
+                continue
+            m, v, u, _ = metric_of(r, r["ms_per_step"])
+            others.append({"workload": name, "metric": m, "value": round(v, 3), "unit": u,
+                           "ms_per_step": round(r["ms_per_step"], 5), "launch_mode": r["launch_mode"],
+                           "active_experts_per_step": r["active_experts_per_step"], "roofline": roofline(r)})
+            del r
+            torch.cuda.empty_cache()
+
+    if rank == 0:
+        shape, T = res["shape"], res["T"]
+        line = {
+            "metric": metric, "value": round(value, 4), "unit": unit, "n_gpus": world, "steps": res["steps"],
+            "warmup": a.warmup, "ms_per_step": round(ms_per_step, 6), "higher_is_better": hib, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 weights/activations, f32 accumulate", "data": "synthetic",
+            "config": {"workload": a.workload, "shape": W.describe(shape), "T": T,
+                       "launch_mode": res["launch_mode"], "ring_layers": res["ring_layers"],
+                       "l2": "inputs larger than L2: ring of distinct layers, touched weights >= 4x L2",
+                       "active_experts_per_step": res["active_experts_per_step"],
+                       "parallelism": "replicas only (no collective)" if world > 1 else "1 GPU"},
+            "roofline": roofline(res),
+            "e2e": {"value": round(e2e_val, 4), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(round(res["launches_per_step"] * res["steps"])),
+            "clocks": res["clocks"],
+        }
+        if not a.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(a.workload)
+        if others:
+            line["others"] = others
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
