@@ -85,8 +85,10 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
-// Longest any device-side wait may last before the kernel gives up and flags MOE_ERR_TIMEOUT.
-constexpr uint64_t kWaitBudgetNs = 2000000000ull;
+// Longest any device-side wait may last before the kernel gives up and flags MOE_ERR_TIMEOUT,
+// in SM clock cycles (about two seconds at the boost clock).  clock64() is used because it is cheap to
+// read; %globaltimer is not.
+constexpr long long kWaitBudgetCycles = 4000000000ll;
 
 __device__ __forceinline__ void flag_error(DeviceState* st, unsigned code, unsigned detail) {
   if (atomicCAS(&st->status, 0u, code) == 0u) st->detail = detail;
@@ -122,12 +124,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: false when the budget ran out (the barrier never completed its phase).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (global_timer_ns() - t0 > kWaitBudgetNs) return false;
+    if (clock64() - t0 > kWaitBudgetCycles) return false;
   }
 }
 
@@ -170,9 +172,10 @@ __device__ __forceinline__ bool grid_barrier(DeviceState* st, unsigned n_ctas, i
       __threadfence();
       st_release(&st->bar_gen, gen + 1u);
     } else {
-      const uint64_t t0 = global_timer_ns();
+      const long long t0 = clock64();
+      unsigned spins = 0;
       while (ld_acquire(&st->bar_gen) == gen) {
-        if (global_timer_ns() - t0 > kWaitBudgetNs) {
+        if ((++spins & 255u) == 0u && clock64() - t0 > kWaitBudgetCycles) {
           ok = 0;
           break;
         }

@@ -5,8 +5,8 @@
 namespace cosmoe {
 
 // ------------------------------------------------------------------------------------ router
-// One warp per token.  Lanes split the d axis; every lane keeps E partial logits, a shuffle
-// tree finishes them, lane 0 does the E-wide softmax / top-k serially (E <= 64).
+// Threads split the d axis and keep E partial logits each; shuffle trees finish them; one warp then
+// does the E-wide softmax and the top-k with one or two experts per lane (E <= 64).
 // Selection runs on the logits: softmax is monotonic, so top_k(W) = top_k(R) (Eq. 2, Eq. 3), and
 // the logits carry more bits than the fp32 probabilities.  Ties go to the lower expert index.
 template <typename XT>
@@ -23,21 +23,55 @@ __device__ __forceinline__ void load_x8<__nv_bfloat16>(const __nv_bfloat16* p, f
 
 constexpr int kRouteWarps = 8;
 
-template <typename XT, int EMAX>
-__global__ void __launch_bounds__(kRouteWarps * 32)
-    route_kernel(const XT* __restrict__ x, const uint16_t* __restrict__ w_router, const float* __restrict__ bias, int T,
-                 int d, int E, int k, int renorm, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
-                 float* __restrict__ probs) {
-  __shared__ float s_logit[kRouteWarps][EMAX];
-  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-  const int t = blockIdx.x * kRouteWarps + wib;
-  if (t >= T) return;
-  float acc[EMAX];
+// Softmax over E logits, top-k and gate weights by one warp: lane l holds logit l (l0) and logit
+// l + 32 (l1).  Ties go to the lower expert index.
+__device__ __forceinline__ void warp_route_finish(float l0, float l1, int E, int k, int renorm, int lane,
+                                                  int32_t* __restrict__ idx_out, float* __restrict__ w_out,
+                                                  float* __restrict__ probs_out) {
+  const float NEG = -3.402823466e38f;
+  const bool has0 = lane < E, has1 = lane + 32 < E;
+  float m = fmaxf(has0 ? l0 : NEG, has1 ? l1 : NEG);
 #pragma unroll
-  for (int e = 0; e < EMAX; ++e) acc[e] = 0.f;
-  const XT* xr = x + (size_t)t * d;
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float p0 = has0 ? expf(l0 - m) : 0.f, p1 = has1 ? expf(l1 - m) : 0.f;
+  const float inv_sum = 1.0f / warp_sum(p0 + p1);
+  if (probs_out) {
+    if (has0) probs_out[lane] = p0 * inv_sum;
+    if (has1) probs_out[lane + 32] = p1 * inv_sum;
+  }
+  bool free0 = has0, free1 = has1;
+  float my_w = 0.f, wtot = 0.f;  // lane j keeps the j-th selected weight
+  int my_idx = 0;
+  for (int j = 0; j < k; ++j) {
+    // this lane's best remaining candidate (its lower index first, so ties keep the lower index)
+    float v = NEG;
+    int id = 0x7fffffff;
+    if (free0) v = l0, id = lane;
+    if (free1 && (!free0 || l1 > v)) v = l1, id = lane + 32;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+      const int oid = __shfl_xor_sync(0xffffffffu, id, o);
+      if (ov > v || (ov == v && oid < id)) v = ov, id = oid;
+    }
+    if (id == lane) free0 = false;
+    if (id == lane + 32) free1 = false;
+    const float pw = expf(v - m) * inv_sum;
+    wtot += pw;
+    if (lane == j) my_w = pw, my_idx = id;
+  }
+  if (lane < k) {
+    idx_out[lane] = my_idx;
+    w_out[lane] = renorm ? my_w / wtot : my_w;
+  }
+}
+
+// Partial logits of one token over the chunks [c_begin, c_end) step c_step of the d axis.
+template <typename XT, int EMAX>
+__device__ __forceinline__ void route_partial(const XT* __restrict__ xr, const uint16_t* __restrict__ w_router, int E,
+                                              int c_begin, int c_end, int c_step, float* acc) {
   const bool vec = (E % 8) == 0;
-  for (int c = lane; c < d / 8; c += 32) {
+  for (int c = c_begin; c < c_end; c += c_step) {
     float xv[8];
     load_x8<XT>(xr + c * 8, xv);
 #pragma unroll
@@ -60,51 +94,92 @@ __global__ void __launch_bounds__(kRouteWarps * 32)
       }
     }
   }
+}
+
+// Many tokens: one warp per token, lanes split the d axis.
+template <typename XT, int EMAX>
+__global__ void __launch_bounds__(kRouteWarps * 32)
+    route_kernel(const XT* __restrict__ x, const uint16_t* __restrict__ w_router, const float* __restrict__ bias, int T,
+                 int d, int E, int k, int renorm, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
+                 float* __restrict__ probs) {
+  __shared__ float s_logit[kRouteWarps][EMAX];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int t = blockIdx.x * kRouteWarps + wib;
+  if (t >= T) return;
+  float acc[EMAX];
+#pragma unroll
+  for (int e = 0; e < EMAX; ++e) acc[e] = 0.f;
+  route_partial<XT, EMAX>(x + (size_t)t * d, w_router, E, lane, d / 8, 32, acc);
 #pragma unroll
   for (int e = 0; e < EMAX; ++e)
     if (e < E) acc[e] = warp_sum(acc[e]);
   if (lane == 0) {
 #pragma unroll
     for (int e = 0; e < EMAX; ++e)
-      if (e < E) s_logit[wib][e] = acc[e] + (bias ? bias[e] : 0.f);
-    float* lg = s_logit[wib];
-    float m = lg[0];
-    for (int e = 1; e < E; ++e) m = fmaxf(m, lg[e]);
-    float sum = 0.f;
-    for (int e = 0; e < E; ++e) sum += expf(lg[e] - m);
-    const float inv_sum = 1.0f / sum;
-    if (probs)
-      for (int e = 0; e < E; ++e) probs[(size_t)t * E + e] = expf(lg[e] - m) * inv_sum;
-    unsigned long long taken = 0ull;
-    float wsel[MOE_MAX_TOPK];
-    float wtot = 0.f;
-    for (int j = 0; j < k; ++j) {
-      int best = -1;
-      float bv = 0.f;
-      for (int e = 0; e < E; ++e) {
-        if ((taken >> e) & 1ull) continue;
-        if (best < 0 || lg[e] > bv) best = e, bv = lg[e];
-      }
-      taken |= 1ull << best;
-      topk_idx[(size_t)t * k + j] = best;
-      wsel[j] = expf(bv - m) * inv_sum;
-      wtot += wsel[j];
-    }
-    const float scale = renorm ? 1.0f / wtot : 1.0f;
-    for (int j = 0; j < k; ++j) topk_w[(size_t)t * k + j] = wsel[j] * scale;
+      if (e < E) s_logit[wib][e] = acc[e];
   }
+  __syncwarp();
+  const float l0 = lane < E ? s_logit[wib][lane] + (bias ? bias[lane] : 0.f) : 0.f;
+  const float l1 = lane + 32 < E ? s_logit[wib][lane + 32] + (bias ? bias[lane + 32] : 0.f) : 0.f;
+  warp_route_finish(l0, l1, E, k, renorm, lane, topk_idx + (size_t)t * k, topk_w + (size_t)t * k,
+                    probs ? probs + (size_t)t * E : nullptr);
+}
+
+// Few tokens (decode): one CTA per token, all 256 threads split the d axis so the weight rows are
+// fetched in a single round trip; warp 0 finishes.
+template <typename XT, int EMAX>
+__global__ void __launch_bounds__(kRouteWarps * 32)
+    route_block_kernel(const XT* __restrict__ x, const uint16_t* __restrict__ w_router, const float* __restrict__ bias,
+                       int T, int d, int E, int k, int renorm, int32_t* __restrict__ topk_idx,
+                       float* __restrict__ topk_w, float* __restrict__ probs) {
+  __shared__ float s_part[kRouteWarps][EMAX];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int t = blockIdx.x;
+  float acc[EMAX];
+#pragma unroll
+  for (int e = 0; e < EMAX; ++e) acc[e] = 0.f;
+  route_partial<XT, EMAX>(x + (size_t)t * d, w_router, E, threadIdx.x, d / 8, kRouteWarps * 32, acc);
+#pragma unroll
+  for (int e = 0; e < EMAX; ++e)
+    if (e < E) acc[e] = warp_sum(acc[e]);
+  if (lane == 0) {
+#pragma unroll
+    for (int e = 0; e < EMAX; ++e)
+      if (e < E) s_part[wib][e] = acc[e];
+  }
+  __syncthreads();
+  if (wib != 0) return;
+  float l0 = 0.f, l1 = 0.f;
+  if (lane < E) {
+    for (int w = 0; w < kRouteWarps; ++w) l0 += s_part[w][lane];
+    if (bias) l0 += bias[lane];
+  }
+  if (lane + 32 < E) {
+    for (int w = 0; w < kRouteWarps; ++w) l1 += s_part[w][lane + 32];
+    if (bias) l1 += bias[lane + 32];
+  }
+  warp_route_finish(l0, l1, E, k, renorm, lane, topk_idx + (size_t)t * k, topk_w + (size_t)t * k,
+                    probs ? probs + (size_t)t * E : nullptr);
 }
 
 template <typename XT>
 static int launch_route_t(moe_ctx* ctx, const void* x, int T, const moe_weights* w, int32_t* idx, float* wt,
                           float* probs, cudaStream_t s) {
   const moe_config& c = ctx->cfg;
-  const dim3 grid((T + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
+  const dim3 block(kRouteWarps * 32);
+  const bool few = T <= 64;
+  const dim3 grid(few ? T : (T + kRouteWarps - 1) / kRouteWarps);
   const XT* xp = (const XT*)x;
   const uint16_t* wr = (const uint16_t*)w->w_router;
-#define ROUTE_CASE(EM)                                                                                               \
-  route_kernel<XT, EM><<<grid, block, 0, s>>>(xp, wr, w->b_router, T, c.d_model, c.n_experts, c.top_k, c.renorm, idx, \
-                                              wt, probs)
+#define ROUTE_CASE(EM)                                                                                              \
+  do {                                                                                                              \
+    if (few)                                                                                                        \
+      route_block_kernel<XT, EM><<<grid, block, 0, s>>>(xp, wr, w->b_router, T, c.d_model, c.n_experts, c.top_k,    \
+                                                        c.renorm, idx, wt, probs);                                  \
+    else                                                                                                            \
+      route_kernel<XT, EM><<<grid, block, 0, s>>>(xp, wr, w->b_router, T, c.d_model, c.n_experts, c.top_k, c.renorm, \
+                                                  idx, wt, probs);                                                  \
+  } while (0)
   if (c.n_experts <= 8)
     ROUTE_CASE(8);
   else if (c.n_experts <= 16)
