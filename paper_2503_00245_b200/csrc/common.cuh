@@ -24,10 +24,13 @@ extern thread_local int g_last_cuda_error;
 
 // Device-resident state of a ctx: status word written by kernels, grid barrier.
 struct DeviceState {
-  unsigned int status;     // 0 ok, else moe_status
-  unsigned int detail;     // where it happened (kernel-specific code)
-  unsigned int bar_count;  // arrivals at the current grid barrier
-  unsigned int bar_gen;    // generation, bumped by the last arriver
+  unsigned int status;  // 0 ok, else moe_status
+  unsigned int detail;  // where it happened (kernel-specific code)
+  unsigned int pad0[30];
+  unsigned int bar_count;  // arrivals at the current grid barrier (own 128-byte line: it takes the atomics)
+  unsigned int pad1[31];
+  unsigned int bar_gen;  // generation, bumped by the last arriver (own line: it takes the polling)
+  unsigned int pad2[31];
 };
 
 }  // namespace cosmoe
@@ -104,6 +107,7 @@ __device__ __forceinline__ void fence_mbar_init() {
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
