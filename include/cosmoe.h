@@ -24,15 +24,19 @@
  *  - Weights are read-only for the library and may be shared between ctxs.
  *  - Shapes: d_model, d_ff and wd_rank multiples of 8; 1 <= top_k <= n_experts <= 64;
  *    top_k <= 8.  Anything else: MOE_ERR_UNSUPPORTED, nothing is read or written.
+ *    The streaming path of dense experts also needs d_model <= 2048.
+ *  - The streaming path sums the CTAs' partial outputs with 64-bit fixed-point atomics
+ *    (2^-36 resolution): integer addition is associative, so results do not depend on
+ *    the order of arrival and repeated calls are bit-identical.
  *
  * Weight layouts.  The mathematical layouts (row-vector convention y = x W) are
  *    w_gate, w_up [E][d][f],  w_down [E][f][d]                       (dense)
  *    gL,uL [E][d][r]  gR,uR [E][r][f]  dL [E][f][r]  dR [E][r][d]    (Eq. 1 factors)
- * The kernels read a packed form in which every output neuron's weights are
- * contiguous (so a slice of an expert is one contiguous run of bytes for the copy
- * engines, and every matrix is K-major for the tensor cores):
- *    gate_up [S][f][2][d] : row c = ( w_gate[:, c] , w_up[:, c] )
- *    down_t  [S][d][f]    : row n = w_down[:, n]
+ * The kernels read a packed form.  Dense experts: everything hidden unit c of an
+ * expert touches is one contiguous run of 3*d values, so any range of hidden units is
+ * one contiguous run of bytes for the copy engines (and for a host->device fetch):
+ *    gud [S][f][3][d] : row c = ( w_gate[:, c] , w_up[:, c] , w_down[c, :] )
+ * Eq. 1 factors: one output neuron's weights contiguous in every matrix:
  *    wd_a [S][r][2][d] = (gL[:,j], uL[:,j]);  wd_b [S][f][2][r] = (gR[:,c], uR[:,c]);
  *    wd_c [S][r][f] = dL[:,j];                wd_d [S][d][r] = dR[:,n]
  * S = number of expert slots (= E unless an offload cache is used).
@@ -81,8 +85,7 @@ typedef struct moe_config {
 typedef struct moe_weights {
   const void* w_router;       /* dev [d][E] bf16                                       */
   const float* b_router;      /* dev [E] fp32 added to the logits, or NULL             */
-  const void* gate_up;        /* dev packed dense, see above (NULL when wd_rank > 0)   */
-  const void* down_t;         /* dev packed dense                                      */
+  const void* gud;            /* dev packed dense, see above (NULL when wd_rank > 0)   */
   const void* wd_a;           /* dev packed Eq. 1 factors (NULL when wd_rank == 0)     */
   const void* wd_b;
   const void* wd_c;
@@ -119,7 +122,7 @@ int moe_launch_count(moe_ctx* ctx, uint64_t* launches);
  * Inputs in the mathematical layouts, outputs in the packed layouts, all dev bf16.
  * n_experts experts are packed into consecutive slots of the outputs.             */
 int moe_pack_dense(int32_t d_model, int32_t d_ff, int32_t n_experts, const void* w_gate, const void* w_up,
-                   const void* w_down, void* gate_up_out, void* down_t_out, void* stream);
+                   const void* w_down, void* gud_out, void* stream);
 int moe_pack_wd(int32_t d_model, int32_t d_ff, int32_t rank, int32_t n_experts, const void* gL, const void* gR,
                 const void* uL, const void* uR, const void* dL, const void* dR, void* wd_a_out, void* wd_b_out,
                 void* wd_c_out, void* wd_d_out, void* stream);
@@ -159,8 +162,7 @@ int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights*
 
 /* ---- host-resident experts (Eq. 8, Section 3.4.2) --------------------------------
  * All experts of n_layers layers live in pinned host memory in packed form
- * (host_experts[layer*E + e] -> one expert: gate_up part then down_t part,
- * slot_bytes in total).  The device holds slots_per_layer slots per layer
+ * (host_experts[layer*E + e] -> one expert in the gud layout, slot_bytes in total).  The device holds slots_per_layer slots per layer
  * (device_slots: dev, n_layers*slots_per_layer*slot_bytes, caller-owned; on creation
  * slot i of every layer is filled with expert i).  With slots_per_layer == top_k the
  * bookkeeping is exactly Eq. 8; with more slots the least recently used expert that

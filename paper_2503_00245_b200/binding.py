@@ -35,7 +35,7 @@ class moe_config(C.Structure):
 
 class moe_weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
-                ("w_router", "b_router", "gate_up", "down_t", "wd_a", "wd_b", "wd_c", "wd_d", "expert_slot")]
+                ("w_router", "b_router", "gud", "wd_a", "wd_b", "wd_c", "wd_d", "expert_slot")]
 
 
 _LIB = None
@@ -49,7 +49,7 @@ _SIGS = {
     "moe_check": (C.c_int, [_P, _P]),
     "moe_workspace_bytes": (C.c_int, [C.POINTER(moe_config), C.c_int32, C.POINTER(C.c_size_t)]),
     "moe_launch_count": (C.c_int, [_P, C.POINTER(C.c_uint64)]),
-    "moe_pack_dense": (C.c_int, [C.c_int32] * 3 + [_P] * 6),
+    "moe_pack_dense": (C.c_int, [C.c_int32] * 3 + [_P] * 5),
     "moe_pack_wd": (C.c_int, [C.c_int32] * 4 + [_P] * 11),
     "moe_route": (C.c_int, [_P, _P, C.c_int32, C.POINTER(moe_weights), _P, _P, _P, _P]),
     "moe_permute": (C.c_int, [_P, _P, C.c_int32, _P, _P, _P, _P]),
@@ -107,10 +107,10 @@ def make_config(d_model, d_ff, n_experts, top_k, wd_rank=0, x_dtype=MOE_BF16, re
     return moe_config(d_model, d_ff, n_experts, top_k, wd_rank, x_dtype, renorm, path)
 
 
-def make_weights(w_router=None, b_router=None, gate_up=None, down_t=None, wd_a=None, wd_b=None, wd_c=None, wd_d=None,
+def make_weights(w_router=None, b_router=None, gud=None, wd_a=None, wd_b=None, wd_c=None, wd_d=None,
                  expert_slot=None) -> moe_weights:
-    w = moe_weights(*[_ptr(t) for t in (w_router, b_router, gate_up, down_t, wd_a, wd_b, wd_c, wd_d, expert_slot)])
-    w._keep = (w_router, b_router, gate_up, down_t, wd_a, wd_b, wd_c, wd_d, expert_slot)  # keep tensors alive
+    w = moe_weights(*[_ptr(t) for t in (w_router, b_router, gud, wd_a, wd_b, wd_c, wd_d, expert_slot)])
+    w._keep = (w_router, b_router, gud, wd_a, wd_b, wd_c, wd_d, expert_slot)  # keep tensors alive
     return w
 
 
@@ -145,9 +145,9 @@ def moe_launch_count(ctx: int) -> int:
     return n.value
 
 
-def moe_pack_dense(d, f, n_experts, w_gate, w_up, w_down, gate_up_out, down_t_out, stream=None):
-    _ok(_lib().moe_pack_dense(d, f, n_experts, _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(gate_up_out),
-                              _ptr(down_t_out), _stream(stream)), "moe_pack_dense")
+def moe_pack_dense(d, f, n_experts, w_gate, w_up, w_down, gud_out, stream=None):
+    _ok(_lib().moe_pack_dense(d, f, n_experts, _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(gud_out),
+                              _stream(stream)), "moe_pack_dense")
 
 
 def moe_pack_wd(d, f, r, n_experts, gL, gR, uL, uR, dL, dR, wd_a, wd_b, wd_c, wd_d, stream=None):

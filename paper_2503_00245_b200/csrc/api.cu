@@ -61,7 +61,7 @@ static int check_weights(const moe_config& c, const moe_weights* w, bool need_ro
   if (need_router && (!w->w_router || misaligned(w->w_router))) return MOE_ERR_INVALID_ARG;
   if (need_experts) {
     if (c.wd_rank == 0) {
-      if (!w->gate_up || !w->down_t || misaligned(w->gate_up) || misaligned(w->down_t)) return MOE_ERR_INVALID_ARG;
+      if (!w->gud || misaligned(w->gud)) return MOE_ERR_INVALID_ARG;
     } else {
       if (!w->wd_a || !w->wd_b || !w->wd_c || !w->wd_d) return MOE_ERR_INVALID_ARG;
       if (misaligned(w->wd_a) || misaligned(w->wd_b) || misaligned(w->wd_c) || misaligned(w->wd_d))
@@ -128,16 +128,23 @@ int moe_create(const moe_config* cfg, moe_ctx** out) {
   c->launches = 0;
   c->d_state = nullptr;
   c->h_state = nullptr;
+  c->acc = nullptr;
+  c->acc_elems = (cfg->wd_rank == 0 && cfg->d_model <= 2048)
+                     ? (size_t)MOE_STREAM_MAX_TOKENS * cfg->top_k * cfg->d_model
+                     : 0;
   cudaError_t e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_state, sizeof(DeviceState));
   if (e == cudaSuccess) e = cudaMemset(c->d_state, 0, sizeof(DeviceState));
   if (e == cudaSuccess) e = cudaMallocHost((void**)&c->h_state, sizeof(DeviceState));
+  if (e == cudaSuccess && c->acc_elems) e = cudaMalloc((void**)&c->acc, c->acc_elems * sizeof(long long));
+  if (e == cudaSuccess && c->acc_elems) e = cudaMemset(c->acc, 0, c->acc_elems * sizeof(long long));
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     (void)cudaGetLastError();
     if (c->d_state) cudaFree(c->d_state);
     if (c->h_state) cudaFreeHost(c->h_state);
+    if (c->acc) cudaFree(c->acc);
     delete c;
     return MOE_ERR_CUDA;
   }
@@ -149,6 +156,7 @@ int moe_destroy(moe_ctx* ctx) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   if (ctx->d_state) cudaFree(ctx->d_state);
   if (ctx->h_state) cudaFreeHost(ctx->h_state);
+  if (ctx->acc) cudaFree(ctx->acc);
   (void)cudaGetLastError();
   delete ctx;
   return MOE_OK;
@@ -162,6 +170,7 @@ int moe_check(moe_ctx* ctx, void* stream) {
   const unsigned st = ctx->h_state->status;
   if (st == 0) return MOE_OK;
   MOE_CUDA_TRY(cudaMemsetAsync(ctx->d_state, 0, sizeof(DeviceState), s));
+  if (ctx->acc) MOE_CUDA_TRY(cudaMemsetAsync(ctx->acc, 0, ctx->acc_elems * sizeof(long long), s));
   MOE_CUDA_TRY(cudaStreamSynchronize(s));
   return st == MOE_ERR_TIMEOUT ? MOE_ERR_TIMEOUT : MOE_ERR_STATE;
 }
@@ -212,6 +221,8 @@ int moe_expert_ffn(moe_ctx* ctx, const void* x, int32_t T, const moe_weights* w,
   cudaStream_t s = (cudaStream_t)stream;
   if (path == MOE_PATH_STREAM) {
     if (T > MOE_STREAM_MAX_TOKENS) return MOE_ERR_UNSUPPORTED;
+    if (ctx->cfg.wd_rank == 0)
+      return launch_dense_stream(ctx, 1, x, T, w, nullptr, nullptr, expert_offsets, perm, nullptr, out_slots, s);
     return launch_stream_ffn(ctx, 1, x, T, w, nullptr, nullptr, expert_offsets, perm, nullptr, out_slots, (char*)ws, L,
                              s);
   }
@@ -241,10 +252,14 @@ int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights*
   char* wsb = (char*)ws;
   int32_t* idx = topk_idx ? topk_idx : (int32_t*)(wsb + L.topk_idx);
   float* wt = topk_w ? topk_w : (float*)(wsb + L.topk_w);
+  if (path == MOE_PATH_STREAM && ctx->cfg.wd_rank == 0 && T == 1)  // the router runs inside the expert kernel
+    return launch_dense_stream(ctx, 0, x, T, w, idx, wt, nullptr, nullptr, y, nullptr, s);
   rc = launch_route(ctx, x, T, w, idx, wt, nullptr, s);
   if (rc != MOE_OK) return rc;
-  if (path == MOE_PATH_STREAM)
+  if (path == MOE_PATH_STREAM) {
+    if (ctx->cfg.wd_rank == 0) return launch_dense_stream(ctx, 0, x, T, w, idx, wt, nullptr, nullptr, y, nullptr, s);
     return launch_stream_ffn(ctx, 0, x, T, w, idx, wt, nullptr, nullptr, y, nullptr, wsb, L, s);
+  }
   int32_t* offsets = (int32_t*)(wsb + L.offsets);
   int32_t* perm = (int32_t*)(wsb + L.perm);
   int32_t* inv = (int32_t*)(wsb + L.inv);

@@ -31,6 +31,8 @@ struct DeviceState {
   unsigned int pad1[31];
   unsigned int bar_gen;  // generation, bumped by the last arriver (own line: it takes the polling)
   unsigned int pad2[31];
+  unsigned int done_count;  // CTAs that have added their partial outputs (dense streaming path)
+  unsigned int pad3[31];
 };
 
 }  // namespace cosmoe
@@ -42,6 +44,8 @@ struct moe_ctx {
   int max_smem_optin;
   cosmoe::DeviceState* d_state;  // device
   cosmoe::DeviceState* h_state;  // pinned host mirror for moe_check
+  long long* acc;                // device: fixed-point output accumulators of the dense streaming path, kept zero
+  size_t acc_elems;              //         between calls by the kernel itself (MOE_STREAM_MAX_TOKENS*top_k*d)
   unsigned long long launches;
 };
 
@@ -73,6 +77,10 @@ int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_s
 int launch_stream_ffn(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, const int32_t* topk_idx,
                       const float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
                       char* ws, const WsLayout& L, cudaStream_t s);
+// Dense experts, streaming path, one kernel (router fused when T == 1 and mode == 0).
+int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
+                        float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
+                        cudaStream_t s);
 // Tensor-core (prefill) path: out_slots from x gathered by perm.
 int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, const int32_t* offsets,
                       const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, cudaStream_t s);
@@ -217,6 +225,50 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
+
+// Softmax over E logits (Eq. 2), top-k (Eq. 3) and gate weights by one warp: lane l holds logit l (l0)
+// and logit l + 32 (l1).  Selection runs on the logits (softmax is monotonic, and the logits carry more
+// bits than fp32 probabilities); ties go to the lower expert index.  Lane j < k writes the j-th choice.
+__device__ __forceinline__ void warp_route_finish(float l0, float l1, int E, int k, int renorm, int lane,
+                                                  int32_t* __restrict__ idx_out, float* __restrict__ w_out,
+                                                  float* __restrict__ probs_out) {
+  const float NEG = -3.402823466e38f;
+  const bool has0 = lane < E, has1 = lane + 32 < E;
+  float m = fmaxf(has0 ? l0 : NEG, has1 ? l1 : NEG);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float p0 = has0 ? expf(l0 - m) : 0.f, p1 = has1 ? expf(l1 - m) : 0.f;
+  const float inv_sum = 1.0f / warp_sum(p0 + p1);
+  if (probs_out) {
+    if (has0) probs_out[lane] = p0 * inv_sum;
+    if (has1) probs_out[lane + 32] = p1 * inv_sum;
+  }
+  bool free0 = has0, free1 = has1;
+  float my_w = 0.f, wtot = 0.f;  // lane j keeps the j-th selected weight
+  int my_idx = 0;
+  for (int j = 0; j < k; ++j) {
+    // this lane's best remaining candidate (its lower index first, so ties keep the lower index)
+    float v = NEG;
+    int id = 0x7fffffff;
+    if (free0) v = l0, id = lane;
+    if (free1 && (!free0 || l1 > v)) v = l1, id = lane + 32;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+      const int oid = __shfl_xor_sync(0xffffffffu, id, o);
+      if (ov > v || (ov == v && oid < id)) v = ov, id = oid;
+    }
+    if (id == lane) free0 = false;
+    if (id == lane + 32) free1 = false;
+    const float pw = expf(v - m) * inv_sum;
+    wtot += pw;
+    if (lane == j) my_w = pw, my_idx = id;
+  }
+  if (lane < k) {
+    idx_out[lane] = my_idx;
+    w_out[lane] = renorm ? my_w / wtot : my_w;
+  }
+}
 
 #endif  // __CUDACC__
 }  // namespace cosmoe

@@ -1,0 +1,618 @@
+// Streaming (decode) path of dense experts: T <= 16 tokens, d_model <= 2048, ONE kernel per layer.
+//
+// The work is bandwidth: every selected expert's weights are read once.  In the packed layout
+// gud[S][f][3][d] all a hidden unit c of an expert needs -- its gate column, its up column and its
+// row of the down matrix -- is one contiguous run of 3*d values, so a CTA that owns a range of hidden
+// units streams one contiguous run of bytes and finishes those units completely:
+//
+//     g_c = x . gate_c,  u_c = x . up_c,  h_c = silu(g_c) * u_c,      y += (gate weight) * h_c * down_c
+//
+// No second phase, no grid-wide barrier: the CTAs' partial y vectors are summed with 64-bit fixed-point
+// atomics (integer addition is associative, so the sum does not depend on arrival order and repeated
+// calls are bit-identical); the CTA that arrives last converts the sum to the output type and leaves
+// the accumulators zero for the next call.
+//
+// (active expert x hidden unit) pairs are split evenly over the CTAs (one per SM).  Inside a CTA:
+//   producer thread   brings stages of 4 hidden units (4 x 3 x d bf16, <= 48 KB) into a ring with one bulk
+//                     asynchronous copy each (TMA without a tensor map), and each pass's token rows of x;
+//   8 consumer warps  per stage: (1) one dot product each (4 units x {gate, up}) against the token(s),
+//                     (2) after an mbarrier, each lane owns 8 output columns and adds the 4 units'
+//                     h_c * down_c into register accumulators; at the end of a pass the accumulators go
+//                     out as atomics.
+// With one token (T == 1, the batch-1 decode case) the router runs in the prologue of every CTA
+// (logits, softmax, top-k, gate weights: Eq. 2, Eq. 3), so the layer is a single launch.
+// Every wait is bounded; an expired wait sets the ctx's status word and the kernel winds down.
+#include "common.cuh"
+
+namespace cosmoe {
+
+namespace {
+
+constexpr int kWarps = 8;  // consumer warps
+constexpr int kProducerWarp = kWarps;
+constexpr int kThreads = (kWarps + 1) * 32;
+constexpr int kConsumerThreads = kWarps * 32;
+constexpr int kRows = 4;       // hidden units per stage: kWarps dot products
+constexpr int kMaxN = 8;       // tokens of one expert handled per pass over its units
+constexpr int kMaxStages = 8;
+constexpr int kXIters = 8;     // 16-byte chunks of x per lane: d <= 2048
+constexpr int kMaxSlots = MOE_STREAM_MAX_TOKENS * MOE_MAX_TOPK;
+constexpr float kFixScale = 68719476736.0f;      // 2^36
+constexpr double kFixInv = 1.0 / 68719476736.0;
+
+struct DenseParams {
+  int T, k, E, d, f, mode, x_is_bf16, renorm, fused_route;
+  const void* x;
+  const uint16_t* w_router;
+  const float* b_router;
+  int32_t* topk_idx;  // mode 0: routing in (fused_route == 0) or out (fused_route == 1, may be null)
+  float* topk_w;
+  const int32_t* offsets;  // mode 1
+  const int32_t* perm;
+  const int32_t* expert_slot;
+  const uint16_t* gud;
+  void* y;
+  float* out_slots;
+  DeviceState* st;
+  long long* acc;
+  int stage_bytes, n_stages, xs_bytes;
+};
+
+struct Smem {
+  uint64_t full[kMaxStages];   // stage landed
+  uint64_t hbar[kMaxStages];   // all dot products of the stage are in `gu`
+  uint64_t freeb[kMaxStages];  // all consumer warps are done with the stage
+  uint64_t xfull[2];           // token rows of a pass landed in xs[0/1]
+  float gu[kMaxStages][kRows * 2][kMaxN];
+  float red[kWarps][MOE_MAX_EXPERTS];
+  int act_e[MOE_MAX_EXPERTS];
+  int act_slot[MOE_MAX_EXPERTS];
+  int act_off[MOE_MAX_EXPERTS + 1];
+  int slot_tok[kMaxSlots];
+  float slot_w[kMaxSlots];
+  int cursor[MOE_MAX_EXPERTS];
+  int stage_e[kMaxSlots];
+  float stage_w[kMaxSlots];
+  int n_act;
+  int last;
+  volatile int abort;
+};
+constexpr int kSmemHeaderBytes = (sizeof(Smem) + 127) / 128 * 128;
+
+struct Pass {
+  int ai, s0, ns, ra, rb;
+};
+struct PassIt {
+  int ai, ai_hi, grp, ngrp, ra, rb;
+  unsigned long long u0, u1;
+};
+
+__device__ __forceinline__ void item_bounds(const Smem& sm, int f, PassIt& g) {
+  const unsigned long long lo = (unsigned long long)g.ai * f, hi = lo + f;
+  const unsigned long long a = g.u0 > lo ? g.u0 : lo, b = g.u1 < hi ? g.u1 : hi;
+  g.ra = (int)(a - lo);
+  g.rb = b > a ? (int)(b - lo) : g.ra;
+  const int ne = sm.act_off[g.ai + 1] - sm.act_off[g.ai];
+  g.ngrp = (ne + kMaxN - 1) / kMaxN;
+  g.grp = 0;
+}
+__device__ __forceinline__ void pass_init(const Smem& sm, int f, PassIt& g) {
+  const unsigned long long U = (unsigned long long)sm.n_act * f;
+  g.u0 = blockIdx.x * U / gridDim.x;
+  g.u1 = (blockIdx.x + 1ull) * U / gridDim.x;
+  g.ra = g.rb = g.grp = g.ngrp = 0;
+  if (g.u1 > g.u0) {
+    g.ai = (int)(g.u0 / f);
+    g.ai_hi = (int)((g.u1 - 1) / f);
+    item_bounds(sm, f, g);
+  } else {
+    g.ai = 0;
+    g.ai_hi = -1;
+  }
+}
+__device__ __forceinline__ bool next_pass(const Smem& sm, int f, PassIt& g, Pass& ps) {
+  for (;;) {
+    if (g.ai > g.ai_hi) return false;
+    if (g.ra >= g.rb || g.grp >= g.ngrp) {
+      g.ai++;
+      if (g.ai <= g.ai_hi) item_bounds(sm, f, g);
+      continue;
+    }
+    const int ne = sm.act_off[g.ai + 1] - sm.act_off[g.ai];
+    ps.ai = g.ai;
+    ps.s0 = g.grp * kMaxN;
+    ps.ns = min(kMaxN, ne - ps.s0);
+    ps.ra = g.ra;
+    ps.rb = g.rb;
+    g.grp++;
+    return true;
+  }
+}
+
+struct RingPos {
+  int slot;
+  unsigned par;
+  int n;
+  __device__ __forceinline__ void advance(int NS) {
+    ++n;
+    if (++slot == NS) slot = 0, par ^= 1u;
+  }
+};
+
+__device__ __forceinline__ void set_abort(DeviceState* st, Smem& sm, unsigned detail) {
+  sm.abort = 1;
+  flag_error(st, MOE_ERR_TIMEOUT, detail);
+}
+
+__device__ __forceinline__ void dot8(const uint4& wv, const float4& a, const float4& b, float& t0, float& t1) {
+  t0 = fmaf(__uint_as_float(wv.x << 16), a.x, t0);
+  t1 = fmaf(__uint_as_float(wv.x & 0xffff0000u), a.y, t1);
+  t0 = fmaf(__uint_as_float(wv.y << 16), a.z, t0);
+  t1 = fmaf(__uint_as_float(wv.y & 0xffff0000u), a.w, t1);
+  t0 = fmaf(__uint_as_float(wv.z << 16), b.x, t0);
+  t1 = fmaf(__uint_as_float(wv.z & 0xffff0000u), b.y, t1);
+  t0 = fmaf(__uint_as_float(wv.w << 16), b.z, t0);
+  t1 = fmaf(__uint_as_float(wv.w & 0xffff0000u), b.w, t1);
+}
+__device__ __forceinline__ float4 bf16x4_lo(const uint4& r) {
+  return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u), __uint_as_float(r.y << 16),
+                     __uint_as_float(r.y & 0xffff0000u));
+}
+__device__ __forceinline__ float4 bf16x4_hi(const uint4& r) {
+  return make_float4(__uint_as_float(r.z << 16), __uint_as_float(r.z & 0xffff0000u), __uint_as_float(r.w << 16),
+                     __uint_as_float(r.w & 0xffff0000u));
+}
+// 8 consecutive elements of a token row of x held in shared memory (bf16 or fp32).
+__device__ __forceinline__ void load_x_chunk(const unsigned char* row, int c, bool bf16, float4& a, float4& b) {
+  if (bf16) {
+    const uint4 r = reinterpret_cast<const uint4*>(row)[c];
+    a = bf16x4_lo(r), b = bf16x4_hi(r);
+  } else {
+    const float4* q = reinterpret_cast<const float4*>(row) + 2 * c;
+    a = q[0], b = q[1];
+  }
+}
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
+
+// One pass of the consumers: units [ra, rb) of one expert for NT tokens (NT == 1: the token row lives
+// in registers; otherwise the rows are read from shared memory for every dot product).
+template <int NT>
+__device__ __forceinline__ bool consume_pass(const DenseParams& P, Smem& sm, const Pass& ps, const unsigned char* ring,
+                                             const unsigned char* xs, RingPos& rp, int warp, int lane) {
+  DeviceState* st = P.st;
+  const int NS = P.n_stages, d = P.d, chunks = d >> 3;
+  const int n = ps.ns;
+  const bool xbf = P.x_is_bf16 != 0;
+  const int xrow_bytes = d * (xbf ? 2 : 4);
+  const int slot0 = sm.act_off[ps.ai] + ps.s0;
+  // output columns this lane owns in step (2): one 8-column chunk
+  const int cw0 = (warp * chunks) / kWarps, cw1 = ((warp + 1) * chunks) / kWarps;
+  const int mychunk = cw0 + lane;
+  const bool owner = mychunk < cw1;
+  const int cclamp = owner ? mychunk : cw0;
+  float acc[NT][8];
+#pragma unroll
+  for (int s = 0; s < NT; ++s)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[s][j] = 0.f;
+  float4 xr[NT == 1 ? kXIters : 1][2];
+  const int cl = chunks - 1;
+  if (NT == 1) {
+#pragma unroll
+    for (int it = 0; it < kXIters; ++it) {
+      load_x_chunk(xs, min(lane + 32 * it, cl), xbf, xr[NT == 1 ? it : 0][0], xr[NT == 1 ? it : 0][1]);
+      if (lane + 32 * it > cl) xr[NT == 1 ? it : 0][0] = xr[NT == 1 ? it : 0][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  // gate weight of each token of the pass (1 when the unweighted per-slot output is asked for)
+  const float myw = (lane < n) ? sm.slot_w[slot0 + lane] : 0.f;
+
+  for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
+    const int nrows = min(kRows, ps.rb - row0);
+    if (!mbar_wait(&sm.full[rp.slot], rp.par)) {
+      if (lane == 0) set_abort(st, sm, 0x310u);
+      return false;
+    }
+    const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * P.stage_bytes);
+    // ---- (1) this warp's dot product: unit (warp >> 1), gate (even warp) or up (odd warp)
+    const int r = warp >> 1;
+    if (r < nrows) {
+      const uint4* wrow = stage + (size_t)(r * 3 + (warp & 1)) * chunks;
+      if (NT == 1) {
+        float a0 = 0.f, a1 = 0.f;
+        {
+          uint4 wv[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) wv[j] = wrow[min(lane + 32 * j, cl)];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dot8(wv[j], xr[NT == 1 ? j : 0][0], xr[NT == 1 ? j : 0][1], a0, a1);
+        }
+        if (chunks > 128) {
+          uint4 wv[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) wv[j] = wrow[min(lane + 32 * (j + 4), cl)];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dot8(wv[j], xr[NT == 1 ? j + 4 : 0][0], xr[NT == 1 ? j + 4 : 0][1], a0, a1);
+        }
+        const float t = warp_sum(a0 + a1);
+        if (lane == 0) sm.gu[rp.slot][warp][0] = t;
+      } else {
+        float a0[NT], a1[NT];
+#pragma unroll
+        for (int s = 0; s < NT; ++s) a0[s] = 0.f, a1[s] = 0.f;
+        for (int c = lane; c < chunks; c += 32) {
+          const uint4 wv = wrow[c];
+#pragma unroll
+          for (int s = 0; s < NT; ++s) {
+            float4 a, b;
+            load_x_chunk(xs + (size_t)(s < n ? s : n - 1) * xrow_bytes, c, xbf, a, b);
+            dot8(wv, a, b, a0[s], a1[s]);
+          }
+        }
+#pragma unroll
+        for (int s = 0; s < NT; ++s) {
+          const float t = warp_sum(a0[s] + a1[s]);
+          if (lane == 0 && s < n) sm.gu[rp.slot][warp][s] = t;
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.hbar[rp.slot]);
+    if (!mbar_wait(&sm.hbar[rp.slot], rp.par)) {
+      if (lane == 0) set_abort(st, sm, 0x311u);
+      return false;
+    }
+    // ---- (2) h_c for (unit, token) pairs, one per lane, then the rank-1 updates of the owned columns
+    float hv = 0.f;
+    {
+      const int rr = lane / n, s = lane - rr * n;
+      const float wsel = __shfl_sync(0xffffffffu, myw, s);
+      if (rr < nrows) {
+        const float g = sm.gu[rp.slot][2 * rr][s], u = sm.gu[rp.slot][2 * rr + 1][s];
+        hv = g / (1.0f + expf(-g)) * u * wsel;
+      }
+    }
+    for (int rr = 0; rr < nrows; ++rr) {
+      const uint4 wv = stage[(size_t)(rr * 3 + 2) * chunks + cclamp];
+      float w[8];
+      unpack8(wv, w);
+#pragma unroll
+      for (int s = 0; s < NT; ++s) {
+        const float h = __shfl_sync(0xffffffffu, hv, rr * n + (s < n ? s : 0));
+        if (s < n) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[s][j] = fmaf(h, w[j], acc[s][j]);
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.freeb[rp.slot]);
+    rp.advance(NS);
+  }
+  // ---- the pass's partial outputs -> fixed-point accumulators in global memory
+  if (owner) {
+#pragma unroll
+    for (int s = 0; s < NT; ++s) {
+      if (s < n) {
+        const int gs = slot0 + s;
+        const int rowi = P.mode == 0 ? sm.slot_tok[gs] : gs;
+        unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) + (size_t)rowi * d + mychunk * 8;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) atomicAdd(dst + j, (unsigned long long)__float2ll_rn(acc[s][j] * kFixScale));
+      }
+    }
+  }
+  return true;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DenseParams P) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
+  unsigned char* ring = smem_raw + kSmemHeaderBytes;
+  unsigned char* xs = ring + (size_t)P.n_stages * P.stage_bytes;  // 2 buffers of xs_bytes
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int NS = P.n_stages;
+  DeviceState* const st = P.st;
+  const int n_pairs = P.T * P.k;
+
+  // ------------------------------------------------------------------ prologue
+  if (tid == kConsumerThreads) {  // the producer thread sets up the barriers
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(&sm.full[i], 1);
+      mbar_init(&sm.hbar[i], kWarps);
+      mbar_init(&sm.freeb[i], kWarps);
+    }
+    mbar_init(&sm.xfull[0], 1);
+    mbar_init(&sm.xfull[1], 1);
+    fence_mbar_init();
+    fence_proxy_async_smem();
+    sm.abort = 0;
+    sm.last = 0;
+  }
+  if (P.fused_route) {
+    // router logits of the single token: every consumer thread takes rows of W_r (row i = the E weights
+    // of input feature i), 8 experts at a time
+    if (warp < kWarps) {
+      const int d = P.d, E = P.E;
+      if ((E & 7) == 0) {
+        for (int e8 = 0; e8 < E; e8 += 8) {
+          float a[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) a[j] = 0.f;
+          for (int i = tid; i < d; i += kConsumerThreads) {
+            const float xv = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[i]) : ((const float*)P.x)[i];
+            float w[8];
+            unpack8(__ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)i * E + e8)), w);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a[j] = fmaf(xv, w[j], a[j]);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float t = warp_sum(a[j]);
+            if (lane == 0) sm.red[warp][e8 + j] = t;
+          }
+        }
+      } else {
+        for (int e = 0; e < E; ++e) {
+          float a = 0.f;
+          for (int i = tid; i < d; i += kConsumerThreads) {
+            const float xv = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[i]) : ((const float*)P.x)[i];
+            a = fmaf(xv, bf16_to_float(__ldg(P.w_router + (size_t)i * E + e)), a);
+          }
+          a = warp_sum(a);
+          if (lane == 0) sm.red[warp][e] = a;
+        }
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      float l0 = 0.f, l1 = 0.f;
+      if (lane < P.E) {
+        for (int w = 0; w < kWarps; ++w) l0 += sm.red[w][lane];
+        if (P.b_router) l0 += P.b_router[lane];
+      }
+      if (lane + 32 < P.E) {
+        for (int w = 0; w < kWarps; ++w) l1 += sm.red[w][lane + 32];
+        if (P.b_router) l1 += P.b_router[lane + 32];
+      }
+      warp_route_finish(l0, l1, P.E, P.k, P.renorm, lane, sm.stage_e, sm.stage_w, nullptr);
+      __syncwarp();
+      if (blockIdx.x == 0 && lane < P.k) {
+        if (P.topk_idx) P.topk_idx[lane] = sm.stage_e[lane];
+        if (P.topk_w) P.topk_w[lane] = sm.stage_w[lane];
+      }
+    }
+  } else if (P.mode == 0 && warp == 0) {
+    for (int p = lane; p < n_pairs; p += 32) {
+      sm.stage_e[p] = P.topk_idx[p];
+      sm.stage_w[p] = P.topk_w[p];
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    // routing products -> active experts and their slots (same numbering as moe_permute)
+    const int n = n_pairs;
+    int na = 0, bad = 0;
+    sm.act_off[0] = 0;
+    if (P.mode == 0) {
+      for (int e = 0; e < P.E; ++e) sm.cursor[e] = 0;
+      for (int p = 0; p < n && !bad; ++p) {
+        const int e = sm.stage_e[p];
+        if (e < 0 || e >= P.E)
+          bad = 1;
+        else
+          sm.cursor[e]++;
+      }
+      int off = 0;
+      for (int e = 0; e < P.E && !bad; ++e) {
+        const int cnt = sm.cursor[e];
+        sm.cursor[e] = off;
+        if (cnt) {
+          sm.act_e[na] = e;
+          sm.act_off[na] = off;
+          ++na;
+          off += cnt;
+        }
+      }
+      sm.act_off[na] = off;
+      for (int p = 0; p < n && !bad; ++p) {
+        const int s = sm.cursor[sm.stage_e[p]]++;
+        sm.slot_tok[s] = p / P.k;
+        sm.slot_w[s] = sm.stage_w[p];
+      }
+    } else {
+      for (int e = 0; e < P.E; ++e) {
+        const int lo = P.offsets[e], hi = P.offsets[e + 1];
+        if (lo < 0 || hi < lo || hi > n) {
+          bad = 1;
+          break;
+        }
+        if (hi > lo) {
+          if (lo != sm.act_off[na]) bad = 1;
+          for (int s = lo; s < hi && !bad; ++s) {
+            const int p = P.perm[s];
+            if (p < 0 || p >= n) {
+              bad = 1;
+              break;
+            }
+            sm.slot_tok[s] = p / P.k;
+            sm.slot_w[s] = 1.0f;
+          }
+          sm.act_e[na] = e;
+          sm.act_off[na + 1] = hi;
+          ++na;
+        }
+      }
+      if (!bad && sm.act_off[na] != n) bad = 1;
+    }
+    for (int a = 0; a < na && !bad; ++a) {
+      const int sl = P.expert_slot ? P.expert_slot[sm.act_e[a]] : sm.act_e[a];
+      if (sl < 0) bad = 1;
+      sm.act_slot[a] = sl < 0 ? 0 : sl;
+    }
+    if (bad) {
+      flag_error(st, MOE_ERR_STATE, 0x300u);
+      na = 0;  // every CTA takes the same decision from the same data: no CTA streams anything
+    }
+    sm.n_act = na;
+  }
+  __syncthreads();
+
+  PassIt pit;
+  pass_init(sm, P.f, pit);
+  Pass ps;
+  RingPos rp{0, 0u, 0};
+
+  if (warp == kProducerWarp) {
+    // ================================================================= producer
+    if (lane != 0) return;
+    const uint32_t row_bytes = (uint32_t)(3 * P.d * 2);
+    const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
+    bool ok = true;
+    int pn = 0, pn_issued = 0;
+    int last_idx[2] = {-1, -1};  // ring index of the last stage of the pass that used xs[b] before
+    int known_free = -1;         // every ring index <= known_free has been released by the consumers
+    unsigned copy_mask = 0;
+    while (ok && next_pass(sm, P.f, pit, ps)) {
+      const int b = pn & 1;
+      if (last_idx[b] > known_free) {
+        const int L = last_idx[b];
+        if (!mbar_wait(&sm.freeb[L % NS], (unsigned)(L / NS) & 1u)) {
+          set_abort(st, sm, 0x331u);
+          ok = false;
+          break;
+        }
+        known_free = L;
+      }
+      // the pass's token rows
+      const int slot0 = sm.act_off[ps.ai] + ps.s0;
+      fence_proxy_async_smem();
+      ++pn_issued;
+      mbar_arrive_expect_tx(&sm.xfull[b], (uint32_t)ps.ns * xrow_bytes);
+      for (int s = 0; s < ps.ns; ++s)
+        bulk_g2s(xs + (size_t)b * P.xs_bytes + (size_t)s * xrow_bytes,
+                 (const unsigned char*)P.x + (size_t)sm.slot_tok[slot0 + s] * xrow_bytes, xrow_bytes, &sm.xfull[b]);
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(P.gud) +
+                                 ((size_t)sm.act_slot[ps.ai] * P.f + ps.ra) * row_bytes;
+      for (int row = ps.ra; row < ps.rb; row += kRows) {
+        const uint32_t bytes = (uint32_t)min(kRows, ps.rb - row) * row_bytes;
+        if (rp.n >= NS) {
+          if (!mbar_wait(&sm.freeb[rp.slot], rp.par ^ 1u)) {
+            set_abort(st, sm, 0x330u);
+            ok = false;
+            break;
+          }
+          known_free = max(known_free, rp.n - NS);
+        }
+        if (sm.abort) {
+          ok = false;
+          break;
+        }
+        fence_proxy_async_smem();
+        mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
+        bulk_g2s(ring + (size_t)rp.slot * P.stage_bytes, src, bytes, &sm.full[rp.slot]);
+        copy_mask |= 1u << rp.slot;
+        src += bytes;
+        rp.advance(NS);
+      }
+      last_idx[b] = rp.n - 1;
+      ++pn;
+    }
+    if (!ok) {
+      // copies already in flight must land before this CTA's shared memory goes away
+      for (int back = 1; back <= NS && back <= rp.n; ++back) {
+        const int j = rp.n - back;
+        if ((copy_mask >> (j % NS)) & 1u) (void)mbar_wait(&sm.full[j % NS], (unsigned)(j / NS) & 1u);
+      }
+      for (int q = max(0, pn_issued - 2); q < pn_issued; ++q) (void)mbar_wait(&sm.xfull[q & 1], (unsigned)(q >> 1) & 1u);
+    }
+    return;
+  }
+
+  // ===================================================================== consumers
+  {
+    bool ok = true;
+    int pn = 0;
+    while (ok && next_pass(sm, P.f, pit, ps)) {
+      const int b = pn & 1;
+      if (!mbar_wait(&sm.xfull[b], (unsigned)(pn >> 1) & 1u)) {
+        if (lane == 0) set_abort(st, sm, 0x312u);
+        ok = false;
+        break;
+      }
+      const unsigned char* xsb = xs + (size_t)b * P.xs_bytes;
+      if (ps.ns == 1)
+        ok = consume_pass<1>(P, sm, ps, ring, xsb, rp, warp, lane);
+      else if (ps.ns == 2)
+        ok = consume_pass<2>(P, sm, ps, ring, xsb, rp, warp, lane);
+      else if (ps.ns <= 4)
+        ok = consume_pass<4>(P, sm, ps, ring, xsb, rp, warp, lane);
+      else
+        ok = consume_pass<8>(P, sm, ps, ring, xsb, rp, warp, lane);
+      ++pn;
+    }
+  }
+  // ------------------------------------------------------------------ all partial sums are out
+  consumer_sync();
+  if (tid == 0) {
+    __threadfence();
+    const unsigned old = atom_add_acq_rel(&st->done_count, 1u);
+    sm.last = (old == gridDim.x - 1u) ? 1 : 0;
+    __threadfence();
+  }
+  consumer_sync();
+  if (sm.last) {
+    // the last CTA to arrive turns the fixed-point sums into the output and leaves zeros behind
+    const int rows = P.mode == 0 ? P.T : n_pairs;
+    const long long total = (long long)rows * P.d;
+    const bool good = ld_acquire(&st->status) == 0u;
+    for (long long i = tid; i < total; i += kConsumerThreads) {
+      const long long v = __ldcg(P.acc + i);
+      P.acc[i] = 0;
+      if (!good) continue;
+      const float fv = (float)((double)v * kFixInv);
+      if (P.mode == 1)
+        P.out_slots[i] = fv;
+      else if (P.x_is_bf16)
+        ((__nv_bfloat16*)P.y)[i] = __float2bfloat16_rn(fv);
+      else
+        ((float*)P.y)[i] = fv;
+    }
+    if (tid == 0) st->done_count = 0u;
+  }
+}
+
+}  // namespace
+
+int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
+                        float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
+                        cudaStream_t s) {
+  const moe_config& c = ctx->cfg;
+  if (c.d_model > 32 * 8 * kXIters || !ctx->acc) return MOE_ERR_UNSUPPORTED;
+  DenseParams P{};
+  P.T = T, P.k = c.top_k, P.E = c.n_experts, P.d = c.d_model, P.f = c.d_ff, P.mode = mode;
+  P.x_is_bf16 = c.x_dtype == MOE_BF16, P.renorm = c.renorm;
+  P.fused_route = (mode == 0 && T == 1) ? 1 : 0;
+  P.x = x, P.w_router = (const uint16_t*)w->w_router, P.b_router = w->b_router;
+  P.topk_idx = topk_idx, P.topk_w = topk_w, P.offsets = offsets, P.perm = perm;
+  P.expert_slot = w->expert_slot, P.gud = (const uint16_t*)w->gud;
+  P.y = y, P.out_slots = out_slots, P.st = ctx->d_state, P.acc = ctx->acc;
+  const int xrow = c.d_model * (P.x_is_bf16 ? 2 : 4);
+  P.xs_bytes = (min(T, kMaxN) * xrow + 127) / 128 * 128;
+  P.stage_bytes = kRows * 3 * c.d_model * 2;  // multiple of 16; the ring base is 128-byte aligned
+  P.stage_bytes = (P.stage_bytes + 127) / 128 * 128;
+  const size_t fixed = 2 * (size_t)P.xs_bytes + kSmemHeaderBytes + 256;
+  const long long avail = (long long)ctx->max_smem_optin - (long long)fixed;
+  if (avail < 2ll * P.stage_bytes) return MOE_ERR_UNSUPPORTED;
+  P.n_stages = (int)min((long long)kMaxStages, avail / P.stage_bytes);
+  const size_t smem = (size_t)P.n_stages * P.stage_bytes + fixed;
+  const int G = ctx->sm_count;
+  MOE_CUDA_TRY(cudaFuncSetAttribute(dense_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dense_stream_kernel<<<G, kThreads, smem, s>>>(P);
+  MOE_CUDA_TRY(cudaGetLastError());
+  ctx->launches++;
+  return MOE_OK;
+}
+
+}  // namespace cosmoe

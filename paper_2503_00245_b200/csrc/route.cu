@@ -23,49 +23,6 @@ __device__ __forceinline__ void load_x8<__nv_bfloat16>(const __nv_bfloat16* p, f
 
 constexpr int kRouteWarps = 8;
 
-// Softmax over E logits, top-k and gate weights by one warp: lane l holds logit l (l0) and logit
-// l + 32 (l1).  Ties go to the lower expert index.
-__device__ __forceinline__ void warp_route_finish(float l0, float l1, int E, int k, int renorm, int lane,
-                                                  int32_t* __restrict__ idx_out, float* __restrict__ w_out,
-                                                  float* __restrict__ probs_out) {
-  const float NEG = -3.402823466e38f;
-  const bool has0 = lane < E, has1 = lane + 32 < E;
-  float m = fmaxf(has0 ? l0 : NEG, has1 ? l1 : NEG);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  const float p0 = has0 ? expf(l0 - m) : 0.f, p1 = has1 ? expf(l1 - m) : 0.f;
-  const float inv_sum = 1.0f / warp_sum(p0 + p1);
-  if (probs_out) {
-    if (has0) probs_out[lane] = p0 * inv_sum;
-    if (has1) probs_out[lane + 32] = p1 * inv_sum;
-  }
-  bool free0 = has0, free1 = has1;
-  float my_w = 0.f, wtot = 0.f;  // lane j keeps the j-th selected weight
-  int my_idx = 0;
-  for (int j = 0; j < k; ++j) {
-    // this lane's best remaining candidate (its lower index first, so ties keep the lower index)
-    float v = NEG;
-    int id = 0x7fffffff;
-    if (free0) v = l0, id = lane;
-    if (free1 && (!free0 || l1 > v)) v = l1, id = lane + 32;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-      const int oid = __shfl_xor_sync(0xffffffffu, id, o);
-      if (ov > v || (ov == v && oid < id)) v = ov, id = oid;
-    }
-    if (id == lane) free0 = false;
-    if (id == lane + 32) free1 = false;
-    const float pw = expf(v - m) * inv_sum;
-    wtot += pw;
-    if (lane == j) my_w = pw, my_idx = id;
-  }
-  if (lane < k) {
-    idx_out[lane] = my_idx;
-    w_out[lane] = renorm ? my_w / wtot : my_w;
-  }
-}
-
 // Partial logits of one token over the chunks [c_begin, c_end) step c_step of the d axis.
 template <typename XT, int EMAX>
 __device__ __forceinline__ void route_partial(const XT* __restrict__ xr, const uint16_t* __restrict__ w_router, int E,
@@ -369,6 +326,18 @@ __global__ void pack_transpose_kernel(const uint16_t* __restrict__ in, uint16_t*
   }
 }
 
+// out[b][c][sub][:] = in[b][c][:]  (rows copied into an interleaved layout, 16 bytes per thread)
+__global__ void pack_rows_kernel(const uint4* __restrict__ in, uint4* __restrict__ out, long long rows, int chunks,
+                                 int nsub, int sub) {
+  const long long total = rows * chunks;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / chunks;
+    const int c = (int)(i - r * chunks);
+    out[(r * nsub + sub) * chunks + c] = in[i];
+  }
+}
+
 static int pack_one(const void* in, void* out, int B, int R, int C, int nsub, int sub, cudaStream_t s) {
   const dim3 grid((C + 31) / 32, (R + 31) / 32, B), block(32, 8);
   if (grid.y > 65535u || grid.z > 65535u) return MOE_ERR_UNSUPPORTED;
@@ -384,13 +353,16 @@ using namespace cosmoe;
 extern "C" {
 
 int moe_pack_dense(int32_t d, int32_t f, int32_t n_experts, const void* w_gate, const void* w_up, const void* w_down,
-                   void* gate_up_out, void* down_t_out, void* stream) {
-  if (d <= 0 || f <= 0 || n_experts <= 0 || !w_gate || !w_up || !w_down || !gate_up_out || !down_t_out)
-    return MOE_ERR_INVALID_ARG;
+                   void* gud_out, void* stream) {
+  if (d <= 0 || f <= 0 || n_experts <= 0 || !w_gate || !w_up || !w_down || !gud_out) return MOE_ERR_INVALID_ARG;
+  if (d % 8 || f % 8) return MOE_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)stream;
-  int rc = pack_one(w_gate, gate_up_out, n_experts, d, f, 2, 0, s);
-  if (rc == MOE_OK) rc = pack_one(w_up, gate_up_out, n_experts, d, f, 2, 1, s);
-  if (rc == MOE_OK) rc = pack_one(w_down, down_t_out, n_experts, f, d, 1, 0, s);
+  int rc = pack_one(w_gate, gud_out, n_experts, d, f, 3, 0, s);
+  if (rc == MOE_OK) rc = pack_one(w_up, gud_out, n_experts, d, f, 3, 1, s);
+  if (rc == MOE_OK) {
+    pack_rows_kernel<<<148 * 8, 256, 0, s>>>((const uint4*)w_down, (uint4*)gud_out, (long long)n_experts * f, d / 8, 3, 2);
+    MOE_CUDA_TRY(cudaGetLastError());
+  }
   return rc;
 }
 

@@ -1,11 +1,9 @@
-// Streaming (decode) path of the expert FFN: T <= 16 tokens.
+// Streaming (decode) path of weight-decomposed experts (Eq. 1): T <= 16 tokens.
 //
-// The work is bandwidth: every selected expert's weights are read once.  All matrices are stored
+// The work is bandwidth: every selected expert's factors are read once.  All matrices are stored
 // with one output neuron's weights contiguous ("rows"), so a phase is "for my rows: dot(row, input
 // vector) for every token routed to that expert".  One cooperative kernel, one CTA per SM:
 //
-//   dense experts   phase 0: gate_up rows  . x        -> h = silu(g) * u      (global, fp32)
-//                   phase 1: down_t rows   . h        -> y (gate-weighted) or out_slots
 //   Eq. 1 factors   phase 0: wd_a rows . x -> t_g,t_u;  phase 1: wd_b rows . t -> h;
 //                   phase 2: wd_c rows . h -> v;        phase 3: wd_d rows . v -> y / out_slots
 //
@@ -728,9 +726,7 @@ int launch_stream_ffn(moe_ctx* ctx, int mode, const void* x, int T, const moe_we
     ph.in_kind = in_kind, ph.epi_kind = epi, ph.in = in, ph.out = out;
   };
   if (r == 0) {
-    P.n_phases = 2;
-    set(0, w->gate_up, f, d, 2, IN_X, EPI_SWIGLU, nullptr, vec_b);
-    set(1, w->down_t, d, f, 1, IN_SLOT, EPI_FINAL, vec_b, nullptr);
+    return MOE_ERR_UNSUPPORTED;  // dense experts stream through launch_dense_stream
   } else {
     P.n_phases = 4;
     set(0, w->wd_a, r, d, 2, IN_X, EPI_PAIR_RAW, nullptr, vec_a);

@@ -10,12 +10,11 @@ from . import binding as B
 
 
 def pack_dense(w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor):
-    """[E,d,f], [E,d,f], [E,f,d] bf16 (maths layout) -> (gate_up [E,f,2,d], down_t [E,d,f])."""
+    """[E,d,f], [E,d,f], [E,f,d] bf16 (maths layout) -> gud [E,f,3,d]."""
     E, d, f = w_gate.shape
-    gate_up = torch.empty((E, f, 2, d), dtype=torch.bfloat16, device=w_gate.device)
-    down_t = torch.empty((E, d, f), dtype=torch.bfloat16, device=w_gate.device)
-    B.moe_pack_dense(d, f, E, w_gate, w_up, w_down, gate_up, down_t)
-    return gate_up, down_t
+    gud = torch.empty((E, f, 3, d), dtype=torch.bfloat16, device=w_gate.device)
+    B.moe_pack_dense(d, f, E, w_gate, w_up, w_down, gud)
+    return gud
 
 
 def pack_wd(gL, gR, uL, uR, dL, dR):
@@ -44,8 +43,7 @@ class MoELayer:
         self.cfg = B.make_config(d_model, d_ff, n_experts, top_k, self.rank,
                                  B.MOE_F32 if x_dtype == torch.float32 else B.MOE_BF16, int(renorm), path)
         if dense is not None:
-            self.weights = B.make_weights(w_router, b_router, gate_up=dense[0], down_t=dense[1],
-                                          expert_slot=expert_slot)
+            self.weights = B.make_weights(w_router, b_router, gud=dense, expert_slot=expert_slot)
         else:
             self.weights = B.make_weights(w_router, b_router, wd_a=wd[0], wd_b=wd[1], wd_c=wd[2], wd_d=wd[3],
                                           expert_slot=expert_slot)

@@ -70,10 +70,10 @@ def test_pack_layouts():
     import paper_2503_00245_b200 as P
     sh = shape(72, 40, E=3)
     t = W.make_experts(sh, device="cuda")
-    gate_up, down_t = P.pack_dense(t["w_gate"], t["w_up"], t["w_down"])
-    assert torch.equal(gate_up[:, :, 0, :], t["w_gate"].transpose(1, 2))
-    assert torch.equal(gate_up[:, :, 1, :], t["w_up"].transpose(1, 2))
-    assert torch.equal(down_t, t["w_down"].transpose(1, 2))
+    gud = P.pack_dense(t["w_gate"], t["w_up"], t["w_down"])
+    assert torch.equal(gud[:, :, 0, :], t["w_gate"].transpose(1, 2))
+    assert torch.equal(gud[:, :, 1, :], t["w_up"].transpose(1, 2))
+    assert torch.equal(gud[:, :, 2, :], t["w_down"])
     t = W.make_experts(shape(72, 40, E=3, r=16), device="cuda")
     a, b, c, d = P.pack_wd(*(t[n] for n in ("gL", "gR", "uL", "uR", "dL", "dR")))
     assert torch.equal(a[:, :, 0, :], t["gL"].transpose(1, 2)) and torch.equal(a[:, :, 1, :], t["uL"].transpose(1, 2))
