@@ -63,6 +63,7 @@ struct Smem {
   uint64_t hbar[kMaxStages];   // all dot products of the stage are in `gu`
   uint64_t freeb[kMaxStages];  // all consumer warps are done with the stage
   uint64_t xfull[2];           // token rows of a pass landed in xs[0/1]
+  uint64_t cbar;               // barrier over the consumer warps
   float gu[kMaxStages][kRows * 2][kMaxN];
   float red[kWarps][MOE_MAX_EXPERTS];
   int act_e[MOE_MAX_EXPERTS];
@@ -173,7 +174,15 @@ __device__ __forceinline__ void load_x_chunk(const unsigned char* row, int c, bo
   }
 }
 
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
+// Barrier over the consumer warps with a bounded wait (an mbarrier, not bar.sync: a warp that gave up on an
+// expired wait elsewhere must not leave the others parked for ever).  `par` is the caller's phase parity.
+__device__ __forceinline__ bool consumer_sync(Smem& sm, unsigned& par, int lane) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(&sm.cbar);
+  const bool ok = mbar_wait_spin(&sm.cbar, par);
+  par ^= 1u;
+  return ok;
+}
 
 // One pass of the consumers: units [ra, rb) of one expert for NT tokens (NT == 1: the token row lives
 // in registers; otherwise the rows are read from shared memory for every dot product).
@@ -259,11 +268,14 @@ __device__ __forceinline__ bool consume_pass(const DenseParams& P, Smem& sm, con
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.hbar[rp.slot]);
-    if (!mbar_wait(&sm.hbar[rp.slot], rp.par)) {
+    if (!mbar_wait_spin(&sm.hbar[rp.slot], rp.par)) {
       if (lane == 0) set_abort(st, sm, 0x311u);
       return false;
     }
     // ---- (2) h_c for (unit, token) pairs, one per lane, then the rank-1 updates of the owned columns
+    uint4 dw[kRows];
+#pragma unroll
+    for (int rr = 0; rr < kRows; ++rr) dw[rr] = stage[(size_t)(min(rr, nrows - 1) * 3 + 2) * chunks + cclamp];
     float hv = 0.f;
     {
       const int rr = lane / n, s = lane - rr * n;
@@ -273,14 +285,14 @@ __device__ __forceinline__ bool consume_pass(const DenseParams& P, Smem& sm, con
         hv = g / (1.0f + expf(-g)) * u * wsel;
       }
     }
-    for (int rr = 0; rr < nrows; ++rr) {
-      const uint4 wv = stage[(size_t)(rr * 3 + 2) * chunks + cclamp];
+#pragma unroll
+    for (int rr = 0; rr < kRows; ++rr) {
       float w[8];
-      unpack8(wv, w);
+      unpack8(dw[rr], w);
 #pragma unroll
       for (int s = 0; s < NT; ++s) {
-        const float h = __shfl_sync(0xffffffffu, hv, rr * n + (s < n ? s : 0));
-        if (s < n) {
+        const float h = __shfl_sync(0xffffffffu, hv, min(rr * n + (s < n ? s : 0), 31));
+        if (s < n && rr < nrows) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) acc[s][j] = fmaf(h, w[j], acc[s][j]);
         }
@@ -325,6 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     }
     mbar_init(&sm.xfull[0], 1);
     mbar_init(&sm.xfull[1], 1);
+    mbar_init(&sm.cbar, kWarps);
     fence_mbar_init();
     fence_proxy_async_smem();
     sm.abort = 0;
@@ -336,16 +349,28 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     if (warp < kWarps) {
       const int d = P.d, E = P.E;
       if ((E & 7) == 0) {
+        // this thread's input features (d <= 2048: at most 8), fetched in one round trip
+        float xv[kXIters];
+#pragma unroll
+        for (int j = 0; j < kXIters; ++j) {
+          const int i = min(tid + j * kConsumerThreads, d - 1);
+          xv[j] = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[i]) : ((const float*)P.x)[i];
+          if (tid + j * kConsumerThreads >= d) xv[j] = 0.f;
+        }
         for (int e8 = 0; e8 < E; e8 += 8) {
+          uint4 wr[kXIters];
+#pragma unroll
+          for (int j = 0; j < kXIters; ++j)
+            wr[j] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + j * kConsumerThreads, d - 1) * E + e8));
           float a[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) a[j] = 0.f;
-          for (int i = tid; i < d; i += kConsumerThreads) {
-            const float xv = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[i]) : ((const float*)P.x)[i];
-            float w[8];
-            unpack8(__ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)i * E + e8)), w);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) a[j] = fmaf(xv, w[j], a[j]);
+          for (int j = 0; j < kXIters; ++j) {
+            float w[8];
+            unpack8(wr[j], w);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) a[q] = fmaf(xv[j], w[q], a[q]);
           }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -470,6 +495,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     const uint32_t row_bytes = (uint32_t)(3 * P.d * 2);
     const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
     bool ok = true;
+    const uint64_t stream_policy = l2_policy_evict_first();
     int pn = 0, pn_issued = 0;
     int last_idx[2] = {-1, -1};  // ring index of the last stage of the pass that used xs[b] before
     int known_free = -1;         // every ring index <= known_free has been released by the consumers
@@ -511,7 +537,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
-        bulk_g2s(ring + (size_t)rp.slot * P.stage_bytes, src, bytes, &sm.full[rp.slot]);
+        bulk_g2s_hint(ring + (size_t)rp.slot * P.stage_bytes, src, bytes, &sm.full[rp.slot], stream_policy);
         copy_mask |= 1u << rp.slot;
         src += bytes;
         rp.advance(NS);
@@ -554,15 +580,18 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     }
   }
   // ------------------------------------------------------------------ all partial sums are out
-  consumer_sync();
+  // (after an expired wait the warps may be out of step with this barrier: then it can expire too; the
+  // status word is already set and nobody finalises)
+  unsigned cpar = 0;
+  bool fin = consumer_sync(sm, cpar, lane);
   if (tid == 0) {
     __threadfence();
     const unsigned old = atom_add_acq_rel(&st->done_count, 1u);
     sm.last = (old == gridDim.x - 1u) ? 1 : 0;
     __threadfence();
   }
-  consumer_sync();
-  if (sm.last) {
+  fin = consumer_sync(sm, cpar, lane) && fin;
+  if (fin && sm.last) {
     // the last CTA to arrive turns the fixed-point sums into the output and leaves zeros behind
     const int rows = P.mode == 0 ? P.T : n_pairs;
     const long long total = (long long)rows * P.d;
