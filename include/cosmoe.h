@@ -160,6 +160,26 @@ int moe_combine(moe_ctx* ctx, const float* out_slots, const float* topk_w, const
 int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights* w, void* y, int32_t* topk_idx,
                       float* topk_w, void* ws, size_t ws_bytes, void* stream);
 
+/* The whole layer again, for callers that must not allocate device memory: code that runs where
+ * cudaMalloc is off limits -- a plug-in inside a host application that has handed out all of the GPU's
+ * memory up front, or a real-time loop in which an allocation (a device-wide synchronising call) is not
+ * allowed.  The paper has no counterpart of this call; it is a convenience of this library.
+ * No ctx, no workspace: the scratch moe_create would allocate (fixed-point accumulators, status and
+ * arrival-counter words) is a 257 KiB __device__ array inside the library, which every GPU that loads the
+ * library holds until the process exits.  Limits: dense experts only (wd_rank == 0), d_model <= 2048,
+ * T <= 16, streaming path; beyond them the call returns MOE_ERR_UNSUPPORTED and touches nothing.
+ * T >= 2 also needs topk_idx and topk_w (dev, [T][k]) for the routing; at T == 1 they may be NULL.
+ * The first call on a GPU looks up the array's address (cudaGetSymbolAddress, with that GPU current):
+ * make that first call outside any stream capture.  The call itself uses no cudaMalloc / cudaFree and no
+ * allocating library routine; it enqueues two small memsets and the kernels on `stream`.
+ * All calls on one GPU share the array: it keeps the last call's contents, the call clears what it needs
+ * before launching, and two calls that overlap on the GPU (different streams, or different threads)
+ * race on it -- issue them in one stream or serialise them yourself.
+ * T == 0 does no work: it waits for `stream` and returns what the kernels of earlier calls on this GPU
+ * reported (MOE_OK, MOE_ERR_TIMEOUT or MOE_ERR_STATE), clearing the report.                          */
+int moe_layer_forward_static(const moe_config* cfg, const void* x, int32_t T, const moe_weights* w, void* y,
+                             int32_t* topk_idx, float* topk_w, void* stream);
+
 /* ---- host-resident experts (Eq. 8, Section 3.4.2) --------------------------------
  * All experts of n_layers layers live in pinned host memory in packed form
  * (host_experts[layer*E + e] -> one expert in the gud layout, slot_bytes in total).  The device holds slots_per_layer slots per layer

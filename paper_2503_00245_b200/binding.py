@@ -56,6 +56,7 @@ _SIGS = {
     "moe_expert_ffn": (C.c_int, [_P, _P, C.c_int32, C.POINTER(moe_weights), _P, _P, _P, _P, C.c_size_t, _P]),
     "moe_combine": (C.c_int, [_P, _P, _P, _P, C.c_int32, _P, _P]),
     "moe_layer_forward": (C.c_int, [_P, _P, C.c_int32, C.POINTER(moe_weights), _P, _P, _P, _P, C.c_size_t, _P]),
+    "moe_layer_forward_static": (C.c_int, [C.POINTER(moe_config), _P, C.c_int32, C.POINTER(moe_weights), _P, _P, _P, _P]),
     "moe_offload_create": (C.c_int, [C.POINTER(moe_config), C.c_int32, C.c_int32, C.POINTER(_P), _P, C.c_size_t,
                                      C.POINTER(_P)]),
     "moe_offload_destroy": (C.c_int, [_P]),
@@ -178,6 +179,12 @@ def moe_combine(ctx, out_slots, topk_w, inv, T, y, stream=None):
 def moe_layer_forward(ctx, x, T, w: moe_weights, y, topk_idx=None, topk_w=None, ws=None, stream=None):
     _ok(_lib().moe_layer_forward(ctx, _ptr(x), T, C.byref(w), _ptr(y), _ptr(topk_idx), _ptr(topk_w), _ptr(ws),
                                  ws.numel() * ws.element_size(), _stream(stream)), "moe_layer_forward")
+
+
+def moe_layer_forward_static(cfg: moe_config, x, T, w: moe_weights, y, topk_idx=None, topk_w=None, stream=None) -> int:
+    """The layer without a ctx or workspace (nothing is allocated); returns the status instead of raising."""
+    return _lib().moe_layer_forward_static(C.byref(cfg), _ptr(x), T, C.byref(w), _ptr(y), _ptr(topk_idx),
+                                           _ptr(topk_w), _stream(stream))
 
 
 def moe_expert_replacements(topk_trace, B, T, k, n_experts, h_total_out, stream=None):

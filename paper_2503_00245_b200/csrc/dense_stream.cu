@@ -645,3 +645,100 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
 }
 
 }  // namespace cosmoe
+
+// =====================================================================================================
+// moe_layer_forward_static: the same layer for callers that must not allocate.
+//
+// The streaming kernel above needs scratch in global memory: the 64-bit fixed-point accumulators the CTAs
+// add their partial outputs into, and a few words of state (status, arrival counter).  moe_create gets
+// them from cudaMalloc.  Here they live in a file-scope __device__ array instead, so nothing is allocated,
+// at the price of a fixed maximum problem size and of every call on a GPU sharing the one array.
+// =====================================================================================================
+namespace cosmoe {
+namespace {
+
+constexpr int kStaticMaxTokens = MOE_STREAM_MAX_TOKENS;  // 16
+constexpr int kStaticMaxD = 32 * 8 * kXIters;            // 2048
+constexpr size_t kStaticStateBytes = (sizeof(DeviceState) + 255) / 256 * 256;
+constexpr size_t kStaticAccBytes = (size_t)kStaticMaxTokens * kStaticMaxD * sizeof(long long);  // 256 KiB
+constexpr size_t kStaticBytes = kStaticStateBytes + kStaticAccBytes;
+
+// Held by every GPU that loads the library, until the process exits.  In host code this name is only a
+// handle for cudaGetSymbolAddress; it is not a device address and is never passed to a kernel.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticDevice {
+  int ready;
+  unsigned char* base;  // device address of g_static_scratch on this GPU
+  int sm_count, max_smem_optin;
+};
+StaticDevice g_static_dev[kMaxDevices];
+
+// Once per device, with that device current: resolve the array's device address.
+int static_setup(int dev, StaticDevice** out) {
+  if (dev < 0 || dev >= kMaxDevices) return MOE_ERR_UNSUPPORTED;
+  StaticDevice& sd = g_static_dev[dev];
+  if (!sd.ready) {
+    void* p = nullptr;
+    MOE_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+    MOE_CUDA_TRY(cudaDeviceGetAttribute(&sd.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    MOE_CUDA_TRY(cudaDeviceGetAttribute(&sd.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    sd.base = (unsigned char*)p;
+    sd.ready = 1;
+  }
+  *out = &sd;
+  return MOE_OK;
+}
+
+}  // namespace
+}  // namespace cosmoe
+
+extern "C" int moe_layer_forward_static(const moe_config* cfg, const void* x, int32_t T, const moe_weights* w, void* y,
+                                        int32_t* topk_idx, float* topk_w, void* stream) {
+  using namespace cosmoe;
+  int rc = validate_config(cfg);
+  if (rc != MOE_OK) return rc;
+  if (T < 0) return MOE_ERR_INVALID_ARG;
+  if (cfg->wd_rank != 0 || cfg->d_model > kStaticMaxD || T > kStaticMaxTokens) return MOE_ERR_UNSUPPORTED;
+  int dev = 0;
+  MOE_CUDA_TRY(cudaGetDevice(&dev));
+  StaticDevice* sd = nullptr;
+  rc = static_setup(dev, &sd);
+  if (rc != MOE_OK) return rc;
+  cudaStream_t s = (cudaStream_t)stream;
+  DeviceState* st = reinterpret_cast<DeviceState*>(sd->base);
+  long long* acc = reinterpret_cast<long long*>(sd->base + kStaticStateBytes);
+  if (T == 0) {
+    // status query: what the kernels of earlier calls on this GPU reported
+    DeviceState host{};
+    MOE_CUDA_TRY(cudaMemcpyAsync(&host, st, sizeof(DeviceState), cudaMemcpyDeviceToHost, s));
+    MOE_CUDA_TRY(cudaStreamSynchronize(s));
+    if (host.status == 0) return MOE_OK;
+    MOE_CUDA_TRY(cudaMemsetAsync(st, 0, sizeof(DeviceState), s));
+    MOE_CUDA_TRY(cudaStreamSynchronize(s));
+    return host.status == MOE_ERR_TIMEOUT ? MOE_ERR_TIMEOUT : MOE_ERR_STATE;
+  }
+  if (!x || !y || !w || !w->w_router || !w->gud) return MOE_ERR_INVALID_ARG;
+  if (((uintptr_t)x | (uintptr_t)y | (uintptr_t)w->w_router | (uintptr_t)w->gud) & 15u) return MOE_ERR_INVALID_ARG;
+  if (T > 1 && (!topk_idx || !topk_w)) return MOE_ERR_INVALID_ARG;
+  // The array keeps what the last call left.  A call that ran to its end leaves the accumulators and the
+  // arrival counter at zero, one that was cut short does not: clear the part this call uses, keep the status.
+  MOE_CUDA_TRY(cudaMemsetAsync(&st->done_count, 0, sizeof(unsigned int), s));
+  MOE_CUDA_TRY(cudaMemsetAsync(acc, 0, (size_t)T * cfg->d_model * sizeof(long long), s));
+  moe_ctx tmp{};  // a view, not a context: nothing here owns memory
+  tmp.cfg = *cfg;
+  tmp.cfg.path = MOE_PATH_STREAM;
+  tmp.device = dev;
+  tmp.sm_count = sd->sm_count;
+  tmp.max_smem_optin = sd->max_smem_optin;
+  tmp.d_state = st;
+  tmp.h_state = nullptr;
+  tmp.acc = acc;
+  tmp.acc_elems = kStaticAccBytes / sizeof(long long);
+  if (T > 1) {
+    rc = launch_route(&tmp, x, T, w, topk_idx, topk_w, nullptr, s);
+    if (rc != MOE_OK) return rc;
+  }
+  return launch_dense_stream(&tmp, 0, x, T, w, topk_idx, topk_w, nullptr, nullptr, y, nullptr, s);
+}
