@@ -1,11 +1,5 @@
 // Entry points whose kernels are not written yet: they refuse, loudly, rather than fall back.
 #include "common.cuh"
-namespace cosmoe {
-int launch_tensor_ffn(moe_ctx*, const void*, int, const moe_weights*, const int32_t*, const int32_t*, char*,
-                      const WsLayout&, float*, cudaStream_t) {
-  return MOE_ERR_UNSUPPORTED;
-}
-}  // namespace cosmoe
 extern "C" {
 int moe_offload_create(const moe_config*, int32_t, int32_t, const void* const*, void*, size_t, moe_offload**) { return MOE_ERR_UNSUPPORTED; }
 int moe_offload_destroy(moe_offload*) { return MOE_ERR_UNSUPPORTED; }
