@@ -4,4 +4,4 @@
 a context and its workspace) that callers and the benchmark use.
 """
 from . import binding  # noqa: F401
-from .layer import MoELayer, pack_dense, pack_wd  # noqa: F401
+from .layer import MoELayer, OffloadedStack, pack_dense, pack_wd  # noqa: F401

@@ -187,6 +187,55 @@ def moe_layer_forward_static(cfg: moe_config, x, T, w: moe_weights, y, topk_idx=
                                            _ptr(topk_w), _stream(stream))
 
 
+def moe_offload_create(cfg: moe_config, n_layers, slots_per_layer, host_expert_ptrs, device_slots, slot_bytes) -> int:
+    """host_expert_ptrs: sequence of n_layers*E host addresses (pinned memory the caller keeps alive)."""
+    arr = (C.c_void_p * len(host_expert_ptrs))(*host_expert_ptrs)
+    h = _P()
+    _ok(_lib().moe_offload_create(C.byref(cfg), n_layers, slots_per_layer, arr, _ptr(device_slots), slot_bytes,
+                                  C.byref(h)), "moe_offload_create")
+    _KEEP[h.value] = arr
+    return h.value
+
+
+_KEEP = {}
+
+
+def moe_offload_destroy(off: int):
+    _KEEP.pop(off, None)
+    _ok(_lib().moe_offload_destroy(off), "moe_offload_destroy")
+
+
+def moe_offload_ensure(off: int, layer: int, topk_idx_host, stream=None):
+    sel = (C.c_int32 * len(topk_idx_host))(*[int(v) for v in topk_idx_host])
+    _ok(_lib().moe_offload_ensure(off, layer, sel, len(topk_idx_host), _stream(stream)), "moe_offload_ensure")
+
+
+def moe_offload_slot_table(off: int, layer: int) -> int:
+    p = _P()
+    _ok(_lib().moe_offload_slot_table(off, layer, C.byref(p)), "moe_offload_slot_table")
+    return p.value
+
+
+def moe_offload_resident(off: int, layer: int, n_slots: int):
+    out = (C.c_int32 * n_slots)()
+    _ok(_lib().moe_offload_resident(off, layer, out), "moe_offload_resident")
+    return list(out)
+
+
+def moe_offload_stats(off: int):
+    a, b, c = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    _ok(_lib().moe_offload_stats(off, C.byref(a), C.byref(b), C.byref(c)), "moe_offload_stats")
+    return {"fetches": a.value, "bytes": b.value, "hits": c.value}
+
+
+def moe_stack_decode_step(off: int, ctx: int, routers, h, n_layers: int, k: int, ws, stream=None):
+    """routers: ctypes array of moe_weights (one per layer).  Returns the [n_layers][k] selection as a list."""
+    trace = (C.c_int32 * (n_layers * k))()
+    _ok(_lib().moe_stack_decode_step(off, ctx, routers, _ptr(h), trace, _ptr(ws), ws.numel() * ws.element_size(),
+                                     _stream(stream)), "moe_stack_decode_step")
+    return [list(trace[l * k:(l + 1) * k]) for l in range(n_layers)]
+
+
 def moe_expert_replacements(topk_trace, B, T, k, n_experts, h_total_out, stream=None):
     _ok(_lib().moe_expert_replacements(_ptr(topk_trace), B, T, k, n_experts, _ptr(h_total_out), _stream(stream)),
         "moe_expert_replacements")

@@ -77,7 +77,8 @@ int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_s
 int launch_stream_ffn(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, const int32_t* topk_idx,
                       const float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
                       char* ws, const WsLayout& L, cudaStream_t s);
-// Dense experts, streaming path, one kernel (router fused when T == 1 and mode == 0).
+// Dense experts, streaming path, one kernel (router fused when T == 1 and mode == 0; mode 2 = mode 0 with the
+// routing always taken from topk_idx / topk_w).
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
                         float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
                         cudaStream_t s);

@@ -619,10 +619,12 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
                         cudaStream_t s) {
   const moe_config& c = ctx->cfg;
   if (c.d_model > 32 * 8 * kXIters || !ctx->acc) return MOE_ERR_UNSUPPORTED;
+  const bool routing_given = (mode == 2);  // mode 2: the whole layer, but with the caller's routing even at T == 1
+  if (routing_given) mode = 0;
   DenseParams P{};
   P.T = T, P.k = c.top_k, P.E = c.n_experts, P.d = c.d_model, P.f = c.d_ff, P.mode = mode;
   P.x_is_bf16 = c.x_dtype == MOE_BF16, P.renorm = c.renorm;
-  P.fused_route = (mode == 0 && T == 1) ? 1 : 0;
+  P.fused_route = (mode == 0 && T == 1 && !routing_given) ? 1 : 0;
   P.x = x, P.w_router = (const uint16_t*)w->w_router, P.b_router = w->b_router;
   P.topk_idx = topk_idx, P.topk_w = topk_w, P.offsets = offsets, P.perm = perm;
   P.expert_slot = w->expert_slot, P.gud = (const uint16_t*)w->gud;

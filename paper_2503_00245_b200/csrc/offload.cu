@@ -1,0 +1,298 @@
+// Host-resident experts (Eq. 8, Section 3.4.2): a per-layer cache of expert slots in device memory, filled
+// from pinned host memory on routing, and the stacked decode step that uses it; plus the replacement metric
+// of Eq. 4-5 on a routing trace.
+//
+// Bookkeeping is host code: per layer an LRU list over C slots; an expert selected in the current step is never
+// the victim; with C == top_k this is exactly the rule of Eq. 8 (bring in what is selected, drop the rest).
+// Evicted experts are dropped -- the host copy is the master -- so only host->device bytes move.
+// Copies run on the object's own stream: it first waits for the compute stream (nobody may still be reading
+// the victim's slot), copies the expert in chunks, updates the layer's expert->slot table in stream order, and
+// the compute stream then waits for the copy stream's event.
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+struct moe_offload {
+  moe_config cfg;
+  int n_layers, slots, E;
+  const void* const* host_experts;
+  unsigned char* device_slots;
+  size_t slot_bytes;
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_compute, ev_copy;
+  std::vector<std::vector<int>> recency;    // per layer: resident experts, least recently used first
+  std::vector<std::vector<int>> slot_of;    // per layer: expert -> slot or -1
+  int32_t* d_tables;                        // device [n_layers][E]
+  int32_t* h_tables;                        // pinned  [n_layers][E]
+  int32_t* h_route;                         // pinned  [k] routing read-back of the stacked step
+  uint64_t fetches, bytes, hits;
+};
+
+namespace cosmoe {
+namespace {
+
+constexpr size_t kCopyChunk = 8u << 20;  // host->device copies are issued in chunks of this size
+
+// u = h / sqrt(mean(h^2)) -> x (bf16 or fp32); one CTA
+__global__ void rms_glue_kernel(const float* __restrict__ h, int d, void* __restrict__ x, int x_is_bf16) {
+  __shared__ float s_part[32];
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) ss = fmaf(h[i], h[i], ss);
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += s_part[w];
+  const float inv = rsqrtf(tot / (float)d);
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = h[i] * inv;
+    if (x_is_bf16)
+      ((__nv_bfloat16*)x)[i] = __float2bfloat16_rn(v);
+    else
+      ((float*)x)[i] = v;
+  }
+}
+// h += y
+__global__ void residual_kernel(float* __restrict__ h, const void* __restrict__ y, int d, int y_is_bf16) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < d) h[i] += y_is_bf16 ? __bfloat162float(((const __nv_bfloat16*)y)[i]) : ((const float*)y)[i];
+}
+
+// Eq. 4: H = sum_b sum_t sum_e |[e in S(b,t+1)] - [e in S(b,t)]| = size of the symmetric difference of
+// consecutive selections, summed.
+__global__ void replacements_kernel(const int32_t* __restrict__ trace, int B, int T, int k,
+                                    unsigned long long* __restrict__ out) {
+  unsigned long long local = 0;
+  const long long pairs = (long long)B * (T - 1);
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < pairs;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long b = i / (T - 1), t = i % (T - 1);
+    const int32_t* s0 = trace + (b * T + t) * k;
+    const int32_t* s1 = s0 + k;
+    int common = 0;
+    for (int a = 0; a < k; ++a)
+      for (int c = 0; c < k; ++c) common += (s0[a] == s1[c]);
+    local += (unsigned long long)(2 * (k - common));
+  }
+  for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
+  if ((threadIdx.x & 31) == 0 && local) atomicAdd(out, local);
+}
+
+}  // namespace
+}  // namespace cosmoe
+
+using namespace cosmoe;
+
+extern "C" {
+
+int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_per_layer,
+                       const void* const* host_experts, void* device_slots, size_t slot_bytes, moe_offload** out) {
+  if (!out) return MOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = validate_config(cfg);
+  if (rc != MOE_OK) return rc;
+  if (n_layers <= 0 || !host_experts || !device_slots || ((uintptr_t)device_slots & 15u)) return MOE_ERR_INVALID_ARG;
+  if (cfg->wd_rank != 0) return MOE_ERR_UNSUPPORTED;
+  if (slots_per_layer < cfg->top_k || slots_per_layer > cfg->n_experts) return MOE_ERR_INVALID_ARG;
+  if (slot_bytes != (size_t)cfg->d_ff * 3 * cfg->d_model * 2) return MOE_ERR_INVALID_ARG;
+  moe_offload* o = new (std::nothrow) moe_offload();
+  if (!o) return MOE_ERR_STATE;
+  o->cfg = *cfg;
+  o->n_layers = n_layers, o->slots = slots_per_layer, o->E = cfg->n_experts;
+  o->host_experts = host_experts;
+  o->device_slots = (unsigned char*)device_slots;
+  o->slot_bytes = slot_bytes;
+  o->fetches = o->bytes = o->hits = 0;
+  o->copy_stream = nullptr, o->ev_compute = nullptr, o->ev_copy = nullptr;
+  o->d_tables = nullptr, o->h_tables = nullptr, o->h_route = nullptr;
+  const size_t tb = (size_t)n_layers * o->E * sizeof(int32_t);
+  cudaError_t e = cudaStreamCreateWithFlags(&o->copy_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&o->ev_compute, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&o->ev_copy, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&o->d_tables, tb);
+  if (e == cudaSuccess) e = cudaMallocHost((void**)&o->h_tables, tb);
+  if (e == cudaSuccess) e = cudaMallocHost((void**)&o->h_route, sizeof(int32_t) * MOE_MAX_TOPK);
+  if (e == cudaSuccess) {
+    o->recency.assign(n_layers, std::vector<int>());
+    o->slot_of.assign(n_layers, std::vector<int>(o->E, -1));
+    for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
+      for (int s = 0; s < o->slots && e == cudaSuccess; ++s) {  // slot s starts with expert s, expert 0 oldest
+        o->recency[l].push_back(s);
+        o->slot_of[l][s] = s;
+        e = cudaMemcpyAsync(o->device_slots + ((size_t)l * o->slots + s) * slot_bytes,
+                            host_experts[(size_t)l * o->E + s], slot_bytes, cudaMemcpyHostToDevice, o->copy_stream);
+      }
+      for (int x = 0; x < o->E; ++x) o->h_tables[(size_t)l * o->E + x] = o->slot_of[l][x];
+    }
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(o->d_tables, o->h_tables, tb, cudaMemcpyHostToDevice, o->copy_stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(o->copy_stream);
+  if (e != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    (void)cudaGetLastError();
+    moe_offload_destroy(o);
+    return MOE_ERR_CUDA;
+  }
+  *out = o;
+  return MOE_OK;
+}
+
+int moe_offload_destroy(moe_offload* o) {
+  if (!o) return MOE_ERR_INVALID_ARG;
+  if (o->copy_stream) {
+    cudaStreamSynchronize(o->copy_stream);
+    cudaStreamDestroy(o->copy_stream);
+  }
+  if (o->ev_compute) cudaEventDestroy(o->ev_compute);
+  if (o->ev_copy) cudaEventDestroy(o->ev_copy);
+  if (o->d_tables) cudaFree(o->d_tables);
+  if (o->h_tables) cudaFreeHost(o->h_tables);
+  if (o->h_route) cudaFreeHost(o->h_route);
+  (void)cudaGetLastError();
+  delete o;
+  return MOE_OK;
+}
+
+int moe_offload_ensure(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, void* compute_stream) {
+  if (!o || !sel || layer < 0 || layer >= o->n_layers || n <= 0 || n > o->slots) return MOE_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (sel[i] < 0 || sel[i] >= o->E) return MOE_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (sel[j] == sel[i]) return MOE_ERR_INVALID_ARG;
+  }
+  cudaStream_t cs = (cudaStream_t)compute_stream;
+  std::vector<int>& rec = o->recency[layer];
+  std::vector<int>& slot_of = o->slot_of[layer];
+  bool waited = false, any = false;
+  for (int i = 0; i < n; ++i) {
+    const int e = sel[i];
+    if (slot_of[e] >= 0) {
+      o->hits++;
+      for (size_t p = 0; p < rec.size(); ++p)
+        if (rec[p] == e) {
+          rec.erase(rec.begin() + p);
+          break;
+        }
+      rec.push_back(e);
+      continue;
+    }
+    int victim = -1;
+    size_t vp = 0;
+    for (size_t p = 0; p < rec.size() && victim < 0; ++p) {
+      bool selected = false;
+      for (int j = 0; j < n; ++j) selected |= (sel[j] == rec[p]);
+      if (!selected) victim = rec[p], vp = p;
+    }
+    if (victim < 0) return MOE_ERR_STATE;
+    if (!waited) {  // work already queued on the compute stream may still read the victim's slot
+      MOE_CUDA_TRY(cudaEventRecord(o->ev_compute, cs));
+      MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->ev_compute, 0));
+      waited = true;
+    }
+    const int slot = slot_of[victim];
+    slot_of[victim] = -1;
+    rec.erase(rec.begin() + vp);
+    slot_of[e] = slot;
+    rec.push_back(e);
+    unsigned char* dst = o->device_slots + ((size_t)layer * o->slots + slot) * o->slot_bytes;
+    const unsigned char* src = (const unsigned char*)o->host_experts[(size_t)layer * o->E + e];
+    for (size_t off = 0; off < o->slot_bytes; off += kCopyChunk) {
+      const size_t nb = o->slot_bytes - off < kCopyChunk ? o->slot_bytes - off : kCopyChunk;
+      MOE_CUDA_TRY(cudaMemcpyAsync(dst + off, src + off, nb, cudaMemcpyHostToDevice, o->copy_stream));
+    }
+    o->fetches++;
+    o->bytes += o->slot_bytes;
+    any = true;
+  }
+  if (any) {
+    int32_t* ht = o->h_tables + (size_t)layer * o->E;
+    for (int x = 0; x < o->E; ++x) ht[x] = slot_of[x];
+    MOE_CUDA_TRY(cudaMemcpyAsync(o->d_tables + (size_t)layer * o->E, ht, sizeof(int32_t) * o->E, cudaMemcpyHostToDevice,
+                                 o->copy_stream));
+    MOE_CUDA_TRY(cudaEventRecord(o->ev_copy, o->copy_stream));
+    MOE_CUDA_TRY(cudaStreamWaitEvent(cs, o->ev_copy, 0));
+  }
+  return MOE_OK;
+}
+
+int moe_offload_slot_table(moe_offload* o, int32_t layer, const int32_t** table) {
+  if (!o || !table || layer < 0 || layer >= o->n_layers) return MOE_ERR_INVALID_ARG;
+  *table = o->d_tables + (size_t)layer * o->E;
+  return MOE_OK;
+}
+
+int moe_offload_resident(moe_offload* o, int32_t layer, int32_t* slots_host) {
+  if (!o || !slots_host || layer < 0 || layer >= o->n_layers) return MOE_ERR_INVALID_ARG;
+  for (int e = 0; e < o->E; ++e)
+    if (o->slot_of[layer][e] >= 0) slots_host[o->slot_of[layer][e]] = e;
+  return MOE_OK;
+}
+
+int moe_offload_stats(moe_offload* o, uint64_t* fetches, uint64_t* bytes, uint64_t* hits) {
+  if (!o) return MOE_ERR_INVALID_ARG;
+  if (fetches) *fetches = o->fetches;
+  if (bytes) *bytes = o->bytes;
+  if (hits) *hits = o->hits;
+  return MOE_OK;
+}
+
+int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* routers, float* h, int32_t* trace_host,
+                          void* ws, size_t ws_bytes, void* stream) {
+  if (!o || !ctx || !routers || !h || !ws) return MOE_ERR_INVALID_ARG;
+  const moe_config& c = ctx->cfg;
+  if (c.wd_rank != 0 || c.d_model != o->cfg.d_model || c.d_ff != o->cfg.d_ff || c.n_experts != o->E ||
+      c.top_k != o->cfg.top_k)
+    return MOE_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(c, 1);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  if ((size_t)c.d_ff * c.top_k * 2 < (size_t)c.d_model * 4) return MOE_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)stream;
+  char* wsb = (char*)ws;
+  int32_t* idx = (int32_t*)(wsb + L.topk_idx);
+  float* wt = (float*)(wsb + L.topk_w);
+  void* u = wsb + L.hidden;               // the normalised input of the layer (x dtype; the region is >= 4*d bytes)
+  void* y = wsb + L.out_slots;            // the layer's output (x dtype)
+  const int d = c.d_model, k = c.top_k;
+  const int xbf = c.x_dtype == MOE_BF16;
+  for (int l = 0; l < o->n_layers; ++l) {
+    rms_glue_kernel<<<1, 256, 0, s>>>(h, d, u, xbf);
+    MOE_CUDA_TRY(cudaGetLastError());
+    ctx->launches++;
+    int rc = launch_route(ctx, u, 1, &routers[l], idx, wt, nullptr, s);
+    if (rc != MOE_OK) return rc;
+    // the host issues the copies, so it has to see the selection
+    MOE_CUDA_TRY(cudaMemcpyAsync(o->h_route, idx, sizeof(int32_t) * k, cudaMemcpyDeviceToHost, s));
+    MOE_CUDA_TRY(cudaStreamSynchronize(s));
+    for (int j = 0; j < k; ++j) {
+      if (trace_host) trace_host[(size_t)l * k + j] = o->h_route[j];
+    }
+    rc = moe_offload_ensure(o, l, o->h_route, k, stream);
+    if (rc != MOE_OK) return rc;
+    moe_weights w = routers[l];
+    w.gud = o->device_slots + (size_t)l * o->slots * o->slot_bytes;
+    w.expert_slot = o->d_tables + (size_t)l * o->E;
+    rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, y, nullptr, s);
+    if (rc != MOE_OK) return rc;
+    residual_kernel<<<(d + 255) / 256, 256, 0, s>>>(h, y, d, xbf);
+    MOE_CUDA_TRY(cudaGetLastError());
+    ctx->launches++;
+  }
+  return MOE_OK;
+}
+
+int moe_expert_replacements(const int32_t* trace, int32_t B, int32_t T, int32_t k, int32_t n_experts,
+                            unsigned long long* h_total_out, void* stream) {
+  if (!trace || !h_total_out || B <= 0 || T <= 0 || k <= 0 || k > MOE_MAX_TOPK || n_experts <= 0)
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  MOE_CUDA_TRY(cudaMemsetAsync(h_total_out, 0, sizeof(unsigned long long), s));
+  if (T < 2) return MOE_OK;
+  const long long pairs = (long long)B * (T - 1);
+  const int grid = (int)((pairs + 255) / 256 < 1184 ? (pairs + 255) / 256 : 1184);
+  replacements_kernel<<<grid, 256, 0, s>>>(trace, B, T, k, h_total_out);
+  MOE_CUDA_TRY(cudaGetLastError());
+  return MOE_OK;
+}
+
+}  // extern "C"

@@ -117,3 +117,56 @@ class MoELayer:
             self.close()
         except Exception:
             pass
+
+
+class OffloadedStack:
+    """n_layers stacked MoE layers whose experts live in pinned host memory (packed gud layout); the device
+    keeps `slots` experts per layer.  Owns the pinned master copy, the device slots, a ctx and its workspace."""
+
+    def __init__(self, d_model, d_ff, n_experts, top_k, slots, layers, x_dtype=torch.bfloat16, device="cuda"):
+        """layers: iterable of dicts with w_router, b_router and gud [E,f,3,d] (device tensors, consumed one by one)."""
+        import ctypes
+        self.d, self.f, self.E, self.k, self.slots = d_model, d_ff, n_experts, top_k, slots
+        self.cfg = B.make_config(d_model, d_ff, n_experts, top_k, 0,
+                                 B.MOE_F32 if x_dtype == torch.float32 else B.MOE_BF16, 1, B.MOE_PATH_STREAM)
+        self.slot_bytes = d_ff * 3 * d_model * 2
+        self.host, self.routers_t = [], []
+        ptrs = []
+        for lay in layers:
+            hg = torch.empty(lay["gud"].shape, dtype=torch.bfloat16, pin_memory=True)
+            hg.copy_(lay["gud"])
+            self.host.append(hg)
+            self.routers_t.append((lay["w_router"], lay["b_router"]))
+            ptrs += [hg.data_ptr() + e * self.slot_bytes for e in range(n_experts)]
+        self.n_layers = len(self.host)
+        torch.cuda.synchronize()
+        self.device_slots = torch.empty(self.n_layers * slots * self.slot_bytes, dtype=torch.uint8, device=device)
+        self.off = B.moe_offload_create(self.cfg, self.n_layers, slots, ptrs, self.device_slots, self.slot_bytes)
+        self.ctx = B.moe_create(self.cfg)
+        self.ws = torch.empty(B.moe_workspace_bytes(self.cfg, 1), dtype=torch.uint8, device=device)
+        self.routers = (B.moe_weights * self.n_layers)()
+        for l, (wr, br) in enumerate(self.routers_t):
+            self.routers[l].w_router = wr.data_ptr()
+            self.routers[l].b_router = br.data_ptr() if br is not None else None
+        self._ctypes = ctypes
+
+    def step(self, h):
+        """h: fp32 [d] device tensor, updated in place.  Returns the per-layer selections."""
+        return B.moe_stack_decode_step(self.off, self.ctx, self.routers, h, self.n_layers, self.k, self.ws)
+
+    def stats(self):
+        return B.moe_offload_stats(self.off)
+
+    def resident(self, layer):
+        return B.moe_offload_resident(self.off, layer, self.slots)
+
+    def check(self):
+        return B.moe_check(self.ctx)
+
+    def close(self):
+        if self.off:
+            B.moe_offload_destroy(self.off)
+            self.off = None
+        if self.ctx:
+            B.moe_destroy(self.ctx)
+            self.ctx = None

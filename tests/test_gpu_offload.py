@@ -1,0 +1,119 @@
+"""GPU tests of the host-resident-expert path (Eq. 8) and of the replacement metric (Eq. 4-5)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import exrep_oracle as X
+from oracle import moe_oracle as O
+from oracle import offload_oracle as F
+from synth import workloads as W
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def make_stack(sh, n_layers, slots):
+    import paper_2503_00245_b200 as P
+    layers, host = [], []
+    for l in range(n_layers):
+        t = W.make_layer(sh, 1, device="cuda", layer=l)
+        host.append({k: W.to_host_bits(v) for k, v in t.items() if k != "x"})
+        layers.append({"w_router": t["w_router"], "b_router": t["b_router"],
+                       "gud": P.pack_dense(t["w_gate"], t["w_up"], t["w_down"])})
+    stack = P.OffloadedStack(sh.d_model, sh.d_ff, sh.n_experts, sh.top_k, slots, layers,
+                             x_dtype=torch.bfloat16 if sh.x_dtype == "bf16" else torch.float32)
+    return stack, host
+
+
+@pytest.mark.parametrize("slots", [2, 4])
+def test_stacked_decode_with_offload_matches_checker(slots):
+    sh = W.LayerShape("t", 5, 256, 512, n_experts=8, top_k=2, x_dtype="bf16", bias="zipf")
+    n_layers, steps = 3, 10
+    stack, host = make_stack(sh, n_layers, slots)
+    traces = [[] for _ in range(n_layers)]
+    for step in range(steps):
+        h0 = W.make_x(sh.with_(x_dtype="f32"), 1, device="cuda", step=step)[0].contiguous()
+        h = h0.clone()
+        sel = stack.step(h)
+        torch.cuda.synchronize()
+        assert stack.check() == 0
+        # checker: same chain in fp64, layer by layer, fed the rounding points the kernels have
+        hh = h0.cpu().numpy().astype(np.float64)
+        for l in range(n_layers):
+            u = O.rms_glue(hh[None])[0]
+            u_b = torch.from_numpy(u.astype(np.float32)).to(torch.bfloat16)         # the layer input is bf16
+            xin = W.to_host_bits(u_b[None])
+            ex = {k: v for k, v in host[l].items() if k not in ("w_router", "b_router")}
+            ora = O.layer_forward(xin, host[l]["w_router"], host[l]["b_router"], ex, sh.top_k)
+            tie = O.near_tie_tokens(ora["logits"], sh.top_k, U.TIE_GAP)[0]
+            if not tie:
+                assert sel[l] == ora["topk_idx"][0].tolist(), (step, l, sel[l], ora["topk_idx"][0])
+            else:
+                ora = O.layer_forward(xin, host[l]["w_router"], host[l]["b_router"], ex, sh.top_k,
+                                      forced_topk=np.int32([sel[l]]))
+            y_b = torch.from_numpy(ora["y"][0].astype(np.float32)).to(torch.bfloat16).double().numpy()
+            hh = hh + y_b
+            traces[l].append(sel[l])
+        got = h.cpu().numpy().astype(np.float64)
+        # rounding of u and y to bf16 happens at the same places on both sides; what is left is fp32 vs fp64
+        # arithmetic inside the layers, amplified by at most n_layers
+        U.assert_close_rms(got, hh, tol=U.Y_TOL, what=f"h after step {step}")
+    # bookkeeping: fetches, bytes, hits and the final residents, exactly, on the GPU's own routing
+    st = stack.stats()
+    tot = {"n_fetch": 0, "bytes": 0, "hits": 0}
+    for l in range(n_layers):
+        sim = F.lru_cache_sim(traces[l], sh.n_experts, slots, stack.slot_bytes)
+        for k in tot:
+            tot[k] += sim[k]
+        assert stack.resident(l) == sim["slots"][-1]
+    assert (st["fetches"], st["bytes"], st["hits"]) == (tot["n_fetch"], tot["bytes"], tot["hits"])
+    if slots == sh.top_k:          # capacity k: exactly the rule of Eq. 8
+        for l in range(n_layers):
+            eq8 = F.eq8_policy(traces[l])
+            sim = F.lru_cache_sim(traces[l], sh.n_experts, slots, 1)
+            assert [sorted(e for e, _ in f) for f in sim["fetches"]][1:] == eq8[1:]
+    stack.close()
+
+
+def test_offload_ensure_argument_errors():
+    from paper_2503_00245_b200 import binding as B
+    sh = W.LayerShape("t", 5, 256, 512, n_experts=8, top_k=2)
+    stack, _ = make_stack(sh, 1, 3)
+    for bad in ([0, 0], [0, 8], [-1, 2], [0, 1, 2, 3]):
+        with pytest.raises(B.MoeError) as e:
+            B.moe_offload_ensure(stack.off, 0, bad)
+        assert e.value.status == 1
+    with pytest.raises(B.MoeError):
+        B.moe_offload_ensure(stack.off, 1, [0, 1])
+    stack.close()
+
+
+def test_expert_replacements_kernel_matches_eq4_and_fig5():
+    from paper_2503_00245_b200 import binding as B
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    # the paper's worked example (Fig. 5): rebuild the selections from the activity matrices
+    golden = os.path.join(os.path.dirname(__file__), "golden", "fig5_expert_activity.txt")
+    blocks, cur = {}, None
+    for line in open(golden):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("["):
+            cur = blocks.setdefault(line[1:].split("]")[0], [])
+        else:
+            cur.append([int(v) for v in line.split()])
+    for name, want in (("bles", 11), ("moe", 21)):
+        A = np.array(blocks[name]).T                       # [T, E]
+        S = np.stack([np.flatnonzero(r) for r in A]).astype(np.int32)[None]   # [1, T, 2]
+        B.moe_expert_replacements(torch.from_numpy(S).cuda(), 1, S.shape[1], 2, 8, out)
+        torch.cuda.synchronize()
+        assert int(out.item()) // 2 == want
+    # random traces against the checker
+    for seed, (Bn, T, k, E) in enumerate([(3, 50, 2, 8), (1, 2, 1, 4), (4, 1000, 4, 16)]):
+        S = np.stack([W.sticky_routing_trace(100 + seed * 10 + b, T, E, k, 0.6) for b in range(Bn)])
+        B.moe_expert_replacements(torch.from_numpy(S).cuda(), Bn, T, k, E, out)
+        torch.cuda.synchronize()
+        _, H = X.hard_replacements(X.activity_from_topk(S, E))
+        assert int(out.item()) == H
