@@ -42,8 +42,8 @@ WsLayout ws_layout(const moe_config& c, int T) {
   L.vec_c = take(stream_ok ? n * (size_t)c.wd_rank * 4 : 0);
   L.xperm = take(tensor_ok ? n * (size_t)c.d_model * 2 : 0);
   L.hidden = take(tensor_ok ? n * (size_t)c.d_ff * 2 : 0);
-  L.mid_a = take(tensor_ok ? n * 2 * (size_t)c.wd_rank * 2 : 0);
-  L.mid_b = take(tensor_ok ? n * (size_t)c.wd_rank * 2 : 0);
+  L.mid_a = take(tensor_ok ? n * 4 * (size_t)c.wd_rank * 2 : 0);  // t_g, t_u as hi + lo bf16 pairs
+  L.mid_b = take(tensor_ok ? n * 2 * (size_t)c.wd_rank * 2 : 0);  // v as a hi + lo pair
   L.out_slots = take(n * (size_t)c.d_model * 4);
   L.total = off + A;
   return L;

@@ -41,10 +41,13 @@ struct GGParams {
   int dual_a;    // the second half has its own A operand
   int b_nmajor;  // B is stored [k][n] (n contiguous): the down rows of gud
   int b_sub;     // sub-row of the interleaved matrix that single / N-major tiles read
+  int k_wrap;    // > 0: the B operand's k coordinate wraps at k_wrap (A = [hi | lo] halves of a split operand)
+  int split;     // bf16 epilogues also store the rounding remainder: value = hi + lo, lo at column offset out_off_lo
   int epi;
   void* out;
   long long ld_out;    // elements
   long long out_off2;  // EPI_BF16_PAIR: column offset of the second half
+  long long out_off_lo;  // split: column offset of the remainders
   int n_stages;
   DeviceState* st;
 };
@@ -195,17 +198,18 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
         unsigned char* st_a1 = st_a0 + a_bytes;
         unsigned char* st_b = st_a0 + a_bytes * (P.dual_a ? 2 : 1);
         const int k0 = kb * kBK;
+        const int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
         mbar_arrive_expect_tx(&sm.full[s], tx);
         tma_load_2d(st_a0, &map_a0, k0, m0, &sm.full[s]);
         if (P.dual_a) tma_load_2d(st_a1, &map_a1, k0, m0, &sm.full[s]);
         if (P.b_nmajor) {
           for (int j = 0; j < P.bn / 64; ++j)
-            tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, n0 + 64 * j, P.b_sub, k0, e, &sm.full[s]);
+            tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, n0 + 64 * j, P.b_sub, kB, e, &sm.full[s]);
         } else if (P.pair) {
-          tma_load_4d(st_b, &map_b, k0, 0, n0, e, &sm.full[s]);
-          tma_load_4d(st_b + 128 * kBK * 2, &map_b, k0, 1, n0, e, &sm.full[s]);
+          tma_load_4d(st_b, &map_b, kB, 0, n0, e, &sm.full[s]);
+          tma_load_4d(st_b + 128 * kBK * 2, &map_b, kB, 1, n0, e, &sm.full[s]);
         } else {
-          tma_load_4d(st_b, &map_b, k0, P.b_sub, n0, e, &sm.full[s]);
+          tma_load_4d(st_b, &map_b, kB, P.b_sub, n0, e, &sm.full[s]);
         }
         ++issued;
       }
@@ -296,6 +300,19 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
                 }
                 *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
                 *reinterpret_cast<uint4*>(out + P.out_off2 + c + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
+                if (P.split) {
+                  uint32_t ol[4], pl[4];
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    ol[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
+                                        __uint_as_float(g[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
+                    pl[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]) - __uint_as_float(p[j] << 16),
+                                        __uint_as_float(u[8 * v + 2 * j + 1]) - __uint_as_float(p[j] & 0xffff0000u));
+                  }
+                  *reinterpret_cast<uint4*>(out + P.out_off_lo + c + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                  *reinterpret_cast<uint4*>(out + P.out_off2 + P.out_off_lo + c + 8 * v) =
+                      make_uint4(pl[0], pl[1], pl[2], pl[3]);
+                }
               }
             }
           }
@@ -322,6 +339,14 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
                 for (int j = 0; j < 4; ++j)
                   o[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]), __uint_as_float(a[8 * v + 2 * j + 1]));
                 *reinterpret_cast<uint4*>(out + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
+                if (P.split) {
+                  uint32_t ol[4];
+#pragma unroll
+                  for (int j = 0; j < 4; ++j)
+                    ol[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
+                                        __uint_as_float(a[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
+                  *reinterpret_cast<uint4*>(out + P.out_off_lo + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                }
               }
             }
           }
@@ -442,34 +467,39 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
     P.epi = EPI_F32, P.out = out_slots, P.ld_out = d, P.out_off2 = 0;
     return launch_gg(ctx, ma, ma, mb, P, n_slots, s);
   }
-  void* mid_a = ws + L.mid_a;  // [n_slots][2r]: t_g | t_u
-  void* mid_b = ws + L.mid_b;  // [n_slots][r]
+  // The rank-r intermediates t and v are kept as hi + lo pairs of bf16 (value = hi + lo): the GEMMs that
+  // consume them run over K = 2r with the weight slices repeated, so the intermediates carry ~16 mantissa
+  // bits and the chain's only bf16 roundings are those of the dense path (hidden activations, output).
+  const bool split = (r % kBK) == 0;
+  const int tw = split ? 2 * r : r;  // stored width of one intermediate
+  void* mid_a = ws + L.mid_a;  // [n_slots][2*tw]: t_g (hi | lo) | t_u (hi | lo)
+  void* mid_b = ws + L.mid_b;  // [n_slots][tw]:   v (hi | lo)
   // (1) T = X [gL | uL]
   if ((rc = make_map_a(&ma, xperm, n_slots, d, d)) != MOE_OK) return rc;
   if ((rc = make_map_b(&mb, w->wd_a, d, 2, r, E, kBK, 128)) != MOE_OK) return rc;
   P.K = d, P.n_total = r, P.bn = 128, P.pair = 1, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_BF16_PAIR;
-  P.out = mid_a, P.ld_out = 2 * r, P.out_off2 = r;
+  P.k_wrap = 0, P.split = split, P.out = mid_a, P.ld_out = 2 * tw, P.out_off2 = tw, P.out_off_lo = r;
   if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (2) hidden = silu(Tg gR) * (Tu uR)
-  if ((rc = make_map_a(&ma, mid_a, n_slots, r, 2 * r)) != MOE_OK) return rc;
-  if ((rc = make_map_a(&ma1, (const __nv_bfloat16*)mid_a + r, n_slots, r, 2 * r)) != MOE_OK) return rc;
+  if ((rc = make_map_a(&ma, mid_a, n_slots, tw, 2 * tw)) != MOE_OK) return rc;
+  if ((rc = make_map_a(&ma1, (const __nv_bfloat16*)mid_a + tw, n_slots, tw, 2 * tw)) != MOE_OK) return rc;
   if ((rc = make_map_b(&mb, w->wd_b, r, 2, f, E, kBK, 128)) != MOE_OK) return rc;
-  P.K = r, P.n_total = f, P.bn = 128, P.pair = 1, P.dual_a = 1, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_SWIGLU;
-  P.out = hidden, P.ld_out = f, P.out_off2 = 0;
+  P.K = tw, P.n_total = f, P.bn = 128, P.pair = 1, P.dual_a = 1, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_SWIGLU;
+  P.k_wrap = split ? r : 0, P.split = 0, P.out = hidden, P.ld_out = f, P.out_off2 = 0, P.out_off_lo = 0;
   if ((rc = launch_gg(ctx, ma, ma1, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (3) V = hidden dL
   if ((rc = make_map_a(&ma, hidden, n_slots, f, f)) != MOE_OK) return rc;
   P.bn = pick_bn(r, 256);
   if ((rc = make_map_b(&mb, w->wd_c, f, 1, r, E, kBK, P.bn)) != MOE_OK) return rc;
   P.K = f, P.n_total = r, P.pair = 0, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_BF16;
-  P.out = mid_b, P.ld_out = r, P.out_off2 = 0;
+  P.k_wrap = 0, P.split = split, P.out = mid_b, P.ld_out = tw, P.out_off2 = 0, P.out_off_lo = r;
   if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (4) out_slots = V dR
-  if ((rc = make_map_a(&ma, mid_b, n_slots, r, r)) != MOE_OK) return rc;
+  if ((rc = make_map_a(&ma, mid_b, n_slots, tw, tw)) != MOE_OK) return rc;
   P.bn = pick_bn(d, 256);
   if ((rc = make_map_b(&mb, w->wd_d, r, 1, d, E, kBK, P.bn)) != MOE_OK) return rc;
-  P.K = r, P.n_total = d, P.pair = 0, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_F32;
-  P.out = out_slots, P.ld_out = d, P.out_off2 = 0;
+  P.K = tw, P.n_total = d, P.pair = 0, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_F32;
+  P.k_wrap = split ? r : 0, P.split = 0, P.out = out_slots, P.ld_out = d, P.out_off2 = 0, P.out_off_lo = 0;
   return launch_gg(ctx, ma, ma, mb, P, n_slots, s);
 }
 

@@ -23,6 +23,12 @@ def shape(d, f, E=8, k=2, r=0, xd="bf16", bias="none", cfg_id=8):
     (W.WEARABLE, 8, 0),
     (W.WEARABLE, 512, 0),
     (W.PHONE, 1, 0),
+    (W.PHONE, 2048, 0),                             # full-size prefill, uneven expert load (router bias)
+    (W.PHONE_WD128, 2048, 0),
+    (W.PHONE_WD1024, 2048, 0),
+    (W.PHONE, 16, TENSOR),                          # tensor path with nearly empty 128-row tiles
+    (shape(1440, 3840), 300, TENSOR),               # K not a multiple of 64, ragged groups
+    (shape(136, 200, E=6, k=3), 37, TENSOR),        # tiny widths: K and N tails inside one tile
     (W.PHONE_WD128, 1, 0),
     (W.PHONE_WD1024, 1, 0),
     (W.PHONE_OFFLOAD, 1, 0),                        # E = 16, Zipf bias
