@@ -7,7 +7,9 @@
 //                  (2) O = H Wd                  A = H,           B = down rows of gud (N-major) -> fp32 slots
 //   Eq. 1 factors  (1) T = X [gL | uL]   (2) H = silu(Tg gR) * (Tu uR)   (3) V = H dL   (4) O = V dR
 //
-// One CTA computes one 128-row x (up to 256-column) tile:
+// One CTA computes one tile of up to 256 rows x 256 columns: two 128-row halves with their own accumulators
+// share every B slice (128 flop per operand byte moved from L2, against 85 for a 128-row tile); a tile whose
+// second half would be empty (the ragged end of an expert's rows) runs one half.  Roles:
 //   warp 0     TMA producer: 64-wide K slices of A and B into a ring of shared-memory stages (128-byte swizzle);
 //   warp 1     allocates tensor memory and issues tcgen05.mma (M = 128, N <= 256, K = 16 per instruction) with
 //              fp32 accumulators in TMEM; a commit releases each stage back to the producer;
@@ -26,8 +28,9 @@ namespace {
 constexpr int kBM = 128;  // rows per tile (TMEM lanes)
 constexpr int kBK = 64;   // K elements per stage (128 bytes of bf16 = one swizzle row)
 constexpr int kThreadsGG = 192;
-constexpr int kTmemCols = 256;
+constexpr int kTmemCols = 512;  // two accumulators of 256 columns
 constexpr int kMaxStagesGG = 4;
+constexpr int kTileRows = 2 * kBM;  // rows per tile when the A operand is single (two halves)
 
 enum Epi { EPI_SWIGLU = 0, EPI_BF16_PAIR = 1, EPI_BF16 = 2, EPI_F32 = 3 };
 
@@ -132,9 +135,10 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
     grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                         const __grid_constant__ CUtensorMap map_b, const GGParams P) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  // stage layout: [A0 16 KB][A1 16 KB if dual_a][B 32 KB], all 1024-byte aligned (swizzle atoms)
+  // stage layout: [A 16 KB][A' 16 KB][B 32 KB], all 1024-byte aligned (swizzle atoms).  A' is the second
+  // 128-row half of the tile, or the second operand (dual_a, 128-row tiles)
   const uint32_t a_bytes = kBM * kBK * 2, b_bytes = 256 * kBK * 2;
-  const uint32_t stage_bytes = a_bytes * (P.dual_a ? 2 : 1) + b_bytes;
+  const uint32_t stage_bytes = 2 * a_bytes + b_bytes;
   unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   SmemGG& sm = *reinterpret_cast<SmemGG*>(stages + (size_t)P.n_stages * stage_bytes);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -146,15 +150,17 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
     int t = blockIdx.y;
     for (int i = 0; i < P.E; ++i) {
       const int lo = P.offsets[i], hi = P.offsets[i + 1];
-      const int nt = (hi - lo + kBM - 1) / kBM;
+      const int tile_rows = P.dual_a ? kBM : kTileRows;
+      const int nt = (hi - lo + tile_rows - 1) / tile_rows;
       if (t < nt) {
-        e = i, m0 = lo + t * kBM, m_end = hi;
+        e = i, m0 = lo + t * tile_rows, m_end = hi;
         break;
       }
       t -= nt;
     }
   }
   if (e < 0) return;  // uniform over the CTA
+  const int halves = (!P.dual_a && m_end - m0 > kBM) ? 2 : 1;
   const int n0 = blockIdx.x * P.bn;
   const int num_kb = (P.K + kBK - 1) / kBK;
 
@@ -182,8 +188,8 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
   if (warp == 0) {
     // ================================================================= TMA producer
     if (lane == 0) {
-      const uint32_t tx =
-          a_bytes * (P.dual_a ? 2 : 1) + (P.pair ? 2u * 128u * kBK * 2u : (uint32_t)P.bn * kBK * 2u);
+      const uint32_t tx = a_bytes * (P.dual_a ? 2 : halves) +
+                          (P.pair ? 2u * 128u * kBK * 2u : (uint32_t)P.bn * kBK * 2u);
       int issued = 0;
       bool ok = true;
       for (int kb = 0; kb < num_kb; ++kb) {
@@ -196,12 +202,15 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
         }
         unsigned char* st_a0 = stages + (size_t)s * stage_bytes;
         unsigned char* st_a1 = st_a0 + a_bytes;
-        unsigned char* st_b = st_a0 + a_bytes * (P.dual_a ? 2 : 1);
+        unsigned char* st_b = st_a0 + 2 * a_bytes;
         const int k0 = kb * kBK;
         const int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
         mbar_arrive_expect_tx(&sm.full[s], tx);
         tma_load_2d(st_a0, &map_a0, k0, m0, &sm.full[s]);
-        if (P.dual_a) tma_load_2d(st_a1, &map_a1, k0, m0, &sm.full[s]);
+        if (P.dual_a)
+          tma_load_2d(st_a1, &map_a1, k0, m0, &sm.full[s]);
+        else if (halves == 2)
+          tma_load_2d(st_a1, &map_a0, k0, m0 + kBM, &sm.full[s]);
         if (P.b_nmajor) {
           for (int j = 0; j < P.bn / 64; ++j)
             tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, n0 + 64 * j, P.b_sub, kB, e, &sm.full[s]);
@@ -234,7 +243,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
         tc_fence_after();
         const uint32_t a0 = smem_u32(stages + (size_t)s * stage_bytes);
         const uint32_t a1 = a0 + a_bytes;
-        const uint32_t b = a0 + a_bytes * (P.dual_a ? 2 : 1);
+        const uint32_t b = a0 + 2 * a_bytes;
 #pragma unroll
         for (int kk = 0; kk < kBK / 16; ++kk) {
           const bool acc = (kb > 0) || (kk > 0);
@@ -242,6 +251,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           if (P.b_nmajor) {
             const uint64_t db = smem_desc(b + kk * 2048, 64 * kBK * 2, 1024);
             tc_mma_bf16(tmem, da0, db, idesc_single, acc);
+            if (halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
           } else if (P.dual_a) {
             const uint64_t da1 = smem_desc(a1 + kk * 32, 16, 1024);
             const uint64_t db0 = smem_desc(b + kk * 32, 16, 1024);
@@ -251,6 +261,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           } else {
             const uint64_t db = smem_desc(b + kk * 32, 16, 1024);
             tc_mma_bf16(tmem, da0, db, idesc_single, acc);
+            if (halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
           }
         }
         tc_commit(&sm.empty[s]);  // arrives when the MMAs above have finished reading this stage
@@ -260,12 +271,13 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
   } else {
     // ================================================================= epilogue (warps 2..5)
     const int q = warp & 3;  // TMEM lanes 32q .. 32q+31 are the only ones this warp may read
-    const int row = m0 + 32 * q + lane;
-    const bool row_ok = row < m_end;
     if (mbar_wait(&sm.accum_full, 0)) {
       tc_fence_after();
-      const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16);
       const int ncols = min(P.bn, P.n_total - n0);  // valid columns of this tile (multiple of 8)
+     for (int hf = 0; hf < halves; ++hf) {
+      const int row = m0 + hf * kBM + 32 * q + lane;
+      const bool row_ok = row < m_end;
+      const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(hf * 256);
       if (P.epi == EPI_SWIGLU || P.epi == EPI_BF16_PAIR) {
         __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + n0;
         for (int c = 0; c < P.bn; c += 32) {
@@ -352,6 +364,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           }
         }
       }
+     }
     } else if (lane == 0) {
       flag_error(P.st, MOE_ERR_TIMEOUT, 0x402u);
     }
@@ -418,11 +431,12 @@ int launch_gg(moe_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const 
   const moe_config& c = ctx->cfg;
   P.E = c.n_experts;
   P.st = ctx->d_state;
-  P.n_stages = P.dual_a ? 3 : 4;
-  const size_t stage_bytes = (size_t)kBM * kBK * 2 * (P.dual_a ? 2 : 1) + 256 * kBK * 2;
+  P.n_stages = 3;
+  const size_t stage_bytes = (size_t)kBM * kBK * 2 * 2 + 256 * kBK * 2;
   const size_t smem = P.n_stages * stage_bytes + sizeof(SmemGG) + 1024 + 128;
   if ((long long)smem > ctx->max_smem_optin) return MOE_ERR_UNSUPPORTED;
-  const int m_tiles = (n_slots + kBM - 1) / kBM + c.n_experts;  // upper bound over all groupings
+  const int tile_rows = P.dual_a ? kBM : kTileRows;
+  const int m_tiles = (n_slots + tile_rows - 1) / tile_rows + c.n_experts;  // upper bound over all groupings
   const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
   if (m_tiles > 65535) return MOE_ERR_UNSUPPORTED;
   MOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
