@@ -19,6 +19,8 @@
 // K and N tails are zero-filled by TMA.  All waits are bounded; an expired wait sets the ctx's status word.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace cosmoe {
@@ -44,6 +46,7 @@ struct GGParams {
   int dual_a;    // the second half has its own A operand
   int b_nmajor;  // B is stored [k][n] (n contiguous): the down rows of gud
   int b_sub;     // sub-row of the interleaved matrix that single / N-major tiles read
+  int tile_rows; // rows per tile: 256 (two halves) or 128
   int k_wrap;    // > 0: the B operand's k coordinate wraps at k_wrap (A = [hi | lo] halves of a split operand)
   int split;     // bf16 epilogues also store the rounding remainder: value = hi + lo, lo at column offset out_off_lo
   int epi;
@@ -126,11 +129,37 @@ __device__ __forceinline__ uint32_t instr_desc(int n, bool b_nmajor) {
 struct SmemGG {
   uint64_t full[kMaxStagesGG];
   uint64_t empty[kMaxStagesGG];
-  uint64_t accum_full;
+  uint64_t accum_full;   // all MMAs of the current tile have completed
+  uint64_t accum_empty;  // the epilogue has read the accumulators out of TMEM (4 warps arrive)
   uint32_t tmem_base;
   int abort;
+  int tile_prefix[MOE_MAX_EXPERTS + 1];  // row tiles per expert, exclusive scan
 };
 
+struct Tile {
+  int e, m0, m_end, halves, n0;
+};
+
+// idx-th tile of this launch: row-tile major, column tile minor (CTAs that run side by side share the A rows
+// and sweep the expert's B columns, which then sit in L2 for the expert's other row tiles).
+__device__ __forceinline__ bool decode_tile(const GGParams& P, const SmemGG& sm, int idx, int n_tiles, Tile& t) {
+  const int mt = idx / n_tiles, nt = idx - mt * n_tiles;
+  if (mt >= sm.tile_prefix[P.E]) return false;
+  int e = 0;
+  while (sm.tile_prefix[e + 1] <= mt) ++e;
+  const int tile_rows = P.tile_rows;
+  t.e = e;
+  t.m0 = P.offsets[e] + (mt - sm.tile_prefix[e]) * tile_rows;
+  t.m_end = P.offsets[e + 1];
+  t.halves = (!P.dual_a && tile_rows > kBM && t.m_end - t.m0 > kBM) ? 2 : 1;
+  t.n0 = nt * P.bn;
+  return true;
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
+// Persistent: CTA c takes tiles c, c + gridDim.x, ...; the TMA producer runs ahead into the next tile while
+// the epilogue of the current one drains TMEM.
 __global__ void __launch_bounds__(kThreadsGG, 1)
     grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                         const __grid_constant__ CUtensorMap map_b, const GGParams P) {
@@ -143,33 +172,23 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
   SmemGG& sm = *reinterpret_cast<SmemGG*>(stages + (size_t)P.n_stages * stage_bytes);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NS = P.n_stages;
-
-  // ---- which tile: blockIdx.y-th 128-row tile over all experts, blockIdx.x-th column tile
-  int e = -1, m0 = 0, m_end = 0;
-  {
-    int t = blockIdx.y;
-    for (int i = 0; i < P.E; ++i) {
-      const int lo = P.offsets[i], hi = P.offsets[i + 1];
-      const int tile_rows = P.dual_a ? kBM : kTileRows;
-      const int nt = (hi - lo + tile_rows - 1) / tile_rows;
-      if (t < nt) {
-        e = i, m0 = lo + t * tile_rows, m_end = hi;
-        break;
-      }
-      t -= nt;
-    }
-  }
-  if (e < 0) return;  // uniform over the CTA
-  const int halves = (!P.dual_a && m_end - m0 > kBM) ? 2 : 1;
-  const int n0 = blockIdx.x * P.bn;
   const int num_kb = (P.K + kBK - 1) / kBK;
+  const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
 
   if (tid == 0) {
+    int run = 0;
+    for (int i = 0; i < P.E; ++i) {
+      sm.tile_prefix[i] = run;
+      const int rows = P.offsets[i + 1] - P.offsets[i];
+      run += rows > 0 ? (rows + P.tile_rows - 1) / P.tile_rows : 0;
+    }
+    sm.tile_prefix[P.E] = run;
     for (int i = 0; i < NS; ++i) {
       mbar_init(&sm.full[i], 1);
       mbar_init(&sm.empty[i], 1);
     }
     mbar_init(&sm.accum_full, 1);
+    mbar_init(&sm.accum_empty, 4);
     sm.abort = 0;
     fence_mbar_init();
     fence_proxy_async_smem();
@@ -184,46 +203,48 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
+  Tile t;
 
   if (warp == 0) {
     // ================================================================= TMA producer
     if (lane == 0) {
-      const uint32_t tx = a_bytes * (P.dual_a ? 2 : halves) +
-                          (P.pair ? 2u * 128u * kBK * 2u : (uint32_t)P.bn * kBK * 2u);
-      int issued = 0;
+      int it = 0;  // k-blocks issued so far, over all tiles
       bool ok = true;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % NS;
-        if (kb >= NS && !mbar_wait(&sm.empty[s], ((kb / NS) - 1) & 1)) {
-          flag_error(P.st, MOE_ERR_TIMEOUT, 0x400u);
-          sm.abort = 1;
-          ok = false;
-          break;
+      for (int idx = blockIdx.x; ok && decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x) {
+        const uint32_t tx = a_bytes * (P.dual_a ? 2 : t.halves) +
+                            (P.pair ? 2u * 128u * kBK * 2u : (uint32_t)P.bn * kBK * 2u);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % NS;
+          if (it >= NS && !mbar_wait(&sm.empty[s], ((it / NS) - 1) & 1)) {
+            flag_error(P.st, MOE_ERR_TIMEOUT, 0x400u);
+            sm.abort = 1;
+            ok = false;
+            break;
+          }
+          unsigned char* st_a0 = stages + (size_t)s * stage_bytes;
+          unsigned char* st_a1 = st_a0 + a_bytes;
+          unsigned char* st_b = st_a0 + 2 * a_bytes;
+          const int k0 = kb * kBK;
+          const int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
+          mbar_arrive_expect_tx(&sm.full[s], tx);
+          tma_load_2d(st_a0, &map_a0, k0, t.m0, &sm.full[s]);
+          if (P.dual_a)
+            tma_load_2d(st_a1, &map_a1, k0, t.m0, &sm.full[s]);
+          else if (t.halves == 2)
+            tma_load_2d(st_a1, &map_a0, k0, t.m0 + kBM, &sm.full[s]);
+          if (P.b_nmajor) {
+            for (int j = 0; j < P.bn / 64; ++j)
+              tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, t.n0 + 64 * j, P.b_sub, kB, t.e, &sm.full[s]);
+          } else if (P.pair) {
+            tma_load_4d(st_b, &map_b, kB, 0, t.n0, t.e, &sm.full[s]);
+            tma_load_4d(st_b + 128 * kBK * 2, &map_b, kB, 1, t.n0, t.e, &sm.full[s]);
+          } else {
+            tma_load_4d(st_b, &map_b, kB, P.b_sub, t.n0, t.e, &sm.full[s]);
+          }
         }
-        unsigned char* st_a0 = stages + (size_t)s * stage_bytes;
-        unsigned char* st_a1 = st_a0 + a_bytes;
-        unsigned char* st_b = st_a0 + 2 * a_bytes;
-        const int k0 = kb * kBK;
-        const int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
-        mbar_arrive_expect_tx(&sm.full[s], tx);
-        tma_load_2d(st_a0, &map_a0, k0, m0, &sm.full[s]);
-        if (P.dual_a)
-          tma_load_2d(st_a1, &map_a1, k0, m0, &sm.full[s]);
-        else if (halves == 2)
-          tma_load_2d(st_a1, &map_a0, k0, m0 + kBM, &sm.full[s]);
-        if (P.b_nmajor) {
-          for (int j = 0; j < P.bn / 64; ++j)
-            tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, n0 + 64 * j, P.b_sub, kB, e, &sm.full[s]);
-        } else if (P.pair) {
-          tma_load_4d(st_b, &map_b, kB, 0, n0, e, &sm.full[s]);
-          tma_load_4d(st_b + 128 * kBK * 2, &map_b, kB, 1, n0, e, &sm.full[s]);
-        } else {
-          tma_load_4d(st_b, &map_b, kB, P.b_sub, n0, e, &sm.full[s]);
-        }
-        ++issued;
       }
-      if (!ok) {
-        for (int kb = max(0, issued - NS); kb < issued; ++kb) (void)mbar_wait(&sm.full[kb % NS], (kb / NS) & 1);
+      if (!ok) {  // copies in flight must land before the CTA goes away
+        for (int j = max(0, it - NS); j < it; ++j) (void)mbar_wait(&sm.full[j % NS], (j / NS) & 1);
       }
     }
   } else if (warp == 1) {
@@ -231,142 +252,160 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
     if (lane == 0) {
       const uint32_t idesc_pairhalf = instr_desc(128, false);
       const uint32_t idesc_single = instr_desc(P.pair ? 256 : P.bn, P.b_nmajor != 0);
+      int it = 0, tile_i = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % NS;
-        if (!mbar_wait(&sm.full[s], (kb / NS) & 1)) {
-          flag_error(P.st, MOE_ERR_TIMEOUT, 0x401u);
-          sm.abort = 1;
-          ok = false;
-          break;
-        }
-        tc_fence_after();
-        const uint32_t a0 = smem_u32(stages + (size_t)s * stage_bytes);
-        const uint32_t a1 = a0 + a_bytes;
-        const uint32_t b = a0 + 2 * a_bytes;
-#pragma unroll
-        for (int kk = 0; kk < kBK / 16; ++kk) {
-          const bool acc = (kb > 0) || (kk > 0);
-          const uint64_t da0 = smem_desc(a0 + kk * 32, 16, 1024);
-          if (P.b_nmajor) {
-            const uint64_t db = smem_desc(b + kk * 2048, 64 * kBK * 2, 1024);
-            tc_mma_bf16(tmem, da0, db, idesc_single, acc);
-            if (halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
-          } else if (P.dual_a) {
-            const uint64_t da1 = smem_desc(a1 + kk * 32, 16, 1024);
-            const uint64_t db0 = smem_desc(b + kk * 32, 16, 1024);
-            const uint64_t db1 = smem_desc(b + 128 * kBK * 2 + kk * 32, 16, 1024);
-            tc_mma_bf16(tmem, da0, db0, idesc_pairhalf, acc);
-            tc_mma_bf16(tmem + 128, da1, db1, idesc_pairhalf, acc);
-          } else {
-            const uint64_t db = smem_desc(b + kk * 32, 16, 1024);
-            tc_mma_bf16(tmem, da0, db, idesc_single, acc);
-            if (halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
+      for (int idx = blockIdx.x; ok && decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x, ++tile_i) {
+        if (tile_i > 0) {  // the previous tile's accumulators must have left TMEM
+          if (!mbar_wait(&sm.accum_empty, (tile_i - 1) & 1)) {
+            flag_error(P.st, MOE_ERR_TIMEOUT, 0x403u);
+            sm.abort = 1;
+            ok = false;
+            break;
           }
+          tc_fence_after();
         }
-        tc_commit(&sm.empty[s]);  // arrives when the MMAs above have finished reading this stage
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % NS;
+          if (!mbar_wait(&sm.full[s], (it / NS) & 1)) {
+            flag_error(P.st, MOE_ERR_TIMEOUT, 0x401u);
+            sm.abort = 1;
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(stages + (size_t)s * stage_bytes);
+          const uint32_t a1 = a0 + a_bytes;
+          const uint32_t b = a0 + 2 * a_bytes;
+#pragma unroll
+          for (int kk = 0; kk < kBK / 16; ++kk) {
+            const bool acc = (kb > 0) || (kk > 0);
+            const uint64_t da0 = smem_desc(a0 + kk * 32, 16, 1024);
+            if (P.b_nmajor) {
+              const uint64_t db = smem_desc(b + kk * 2048, 64 * kBK * 2, 1024);
+              tc_mma_bf16(tmem, da0, db, idesc_single, acc);
+              if (t.halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
+            } else if (P.dual_a) {
+              const uint64_t da1 = smem_desc(a1 + kk * 32, 16, 1024);
+              const uint64_t db0 = smem_desc(b + kk * 32, 16, 1024);
+              const uint64_t db1 = smem_desc(b + 128 * kBK * 2 + kk * 32, 16, 1024);
+              tc_mma_bf16(tmem, da0, db0, idesc_pairhalf, acc);
+              tc_mma_bf16(tmem + 128, da1, db1, idesc_pairhalf, acc);
+            } else {
+              const uint64_t db = smem_desc(b + kk * 32, 16, 1024);
+              tc_mma_bf16(tmem, da0, db, idesc_single, acc);
+              if (t.halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
+            }
+          }
+          tc_commit(&sm.empty[s]);  // arrives when the MMAs above have finished reading this stage
+        }
+        if (ok) tc_commit(&sm.accum_full);
       }
-      if (ok) tc_commit(&sm.accum_full);
     }
   } else {
     // ================================================================= epilogue (warps 2..5)
     const int q = warp & 3;  // TMEM lanes 32q .. 32q+31 are the only ones this warp may read
-    if (mbar_wait(&sm.accum_full, 0)) {
+    int tile_i = 0;
+    for (int idx = blockIdx.x; decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x, ++tile_i) {
+      if (!mbar_wait(&sm.accum_full, tile_i & 1)) {
+        if (lane == 0) flag_error(P.st, MOE_ERR_TIMEOUT, 0x402u);
+        break;
+      }
       tc_fence_after();
-      const int ncols = min(P.bn, P.n_total - n0);  // valid columns of this tile (multiple of 8)
-     for (int hf = 0; hf < halves; ++hf) {
-      const int row = m0 + hf * kBM + 32 * q + lane;
-      const bool row_ok = row < m_end;
-      const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(hf * 256);
-      if (P.epi == EPI_SWIGLU || P.epi == EPI_BF16_PAIR) {
-        __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + n0;
-        for (int c = 0; c < P.bn; c += 32) {
-          uint32_t g[32], u[32];
-          tc_ld32(tbase + c, g);
-          tc_ld32(tbase + 128 + c, u);
-          tc_wait_ld();
-          if (!row_ok) continue;
-          if (P.epi == EPI_SWIGLU) {
+      const int ncols = min(P.bn, P.n_total - t.n0);  // valid columns of this tile (multiple of 8)
+      for (int hf = 0; hf < t.halves; ++hf) {
+        const int row = t.m0 + hf * kBM + 32 * q + lane;
+        const bool row_ok = row < t.m_end;
+        const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(hf * 256);
+        if (P.epi == EPI_SWIGLU || P.epi == EPI_BF16_PAIR) {
+          __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + t.n0;
+          for (int c = 0; c < P.bn; c += 32) {
+            uint32_t g[32], u[32];
+            tc_ld32(tbase + c, g);
+            tc_ld32(tbase + 128 + c, u);
+            tc_wait_ld();
+            if (!row_ok) continue;
+            if (P.epi == EPI_SWIGLU) {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (c + 8 * v < ncols) {
-                uint32_t o[4];
+              for (int v = 0; v < 4; ++v) {
+                if (c + 8 * v < ncols) {
+                  uint32_t o[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const float g0 = __uint_as_float(g[8 * v + 2 * j]), g1 = __uint_as_float(g[8 * v + 2 * j + 1]);
-                  const float u0 = __uint_as_float(u[8 * v + 2 * j]), u1 = __uint_as_float(u[8 * v + 2 * j + 1]);
-                  o[j] = pack_bf16x2(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+                  for (int j = 0; j < 4; ++j)
+                    o[j] = pack_bf16x2(
+                        silu_mul(__uint_as_float(g[8 * v + 2 * j]), __uint_as_float(u[8 * v + 2 * j])),
+                        silu_mul(__uint_as_float(g[8 * v + 2 * j + 1]), __uint_as_float(u[8 * v + 2 * j + 1])));
+                  *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
-                *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
               }
-            }
-          } else {
+            } else {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (c + 8 * v < ncols) {
-                uint32_t o[4], p[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  o[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]), __uint_as_float(g[8 * v + 2 * j + 1]));
-                  p[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]), __uint_as_float(u[8 * v + 2 * j + 1]));
-                }
-                *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
-                *reinterpret_cast<uint4*>(out + P.out_off2 + c + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
-                if (P.split) {
-                  uint32_t ol[4], pl[4];
+              for (int v = 0; v < 4; ++v) {
+                if (c + 8 * v < ncols) {
+                  uint32_t o[4], p[4];
 #pragma unroll
                   for (int j = 0; j < 4; ++j) {
-                    ol[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
-                                        __uint_as_float(g[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
-                    pl[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]) - __uint_as_float(p[j] << 16),
-                                        __uint_as_float(u[8 * v + 2 * j + 1]) - __uint_as_float(p[j] & 0xffff0000u));
+                    o[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]), __uint_as_float(g[8 * v + 2 * j + 1]));
+                    p[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]), __uint_as_float(u[8 * v + 2 * j + 1]));
                   }
-                  *reinterpret_cast<uint4*>(out + P.out_off_lo + c + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-                  *reinterpret_cast<uint4*>(out + P.out_off2 + P.out_off_lo + c + 8 * v) =
-                      make_uint4(pl[0], pl[1], pl[2], pl[3]);
+                  *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
+                  *reinterpret_cast<uint4*>(out + P.out_off2 + c + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
+                  if (P.split) {
+                    uint32_t ol[4], pl[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                      ol[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
+                                          __uint_as_float(g[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
+                      pl[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]) - __uint_as_float(p[j] << 16),
+                                          __uint_as_float(u[8 * v + 2 * j + 1]) - __uint_as_float(p[j] & 0xffff0000u));
+                    }
+                    *reinterpret_cast<uint4*>(out + P.out_off_lo + c + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                    *reinterpret_cast<uint4*>(out + P.out_off2 + P.out_off_lo + c + 8 * v) =
+                        make_uint4(pl[0], pl[1], pl[2], pl[3]);
+                  }
                 }
               }
             }
           }
-        }
-      } else {
-        for (int c = 0; c < P.bn; c += 32) {
-          uint32_t a[32];
-          tc_ld32(tbase + c, a);
-          tc_wait_ld();
-          if (!row_ok) continue;
-          if (P.epi == EPI_F32) {
-            float* out = (float*)P.out + (size_t)row * P.ld_out + n0 + c;
+        } else {
+          for (int c = 0; c < P.bn; c += 32) {
+            uint32_t a[32];
+            tc_ld32(tbase + c, a);
+            tc_wait_ld();
+            if (!row_ok) continue;
+            if (P.epi == EPI_F32) {
+              float* out = (float*)P.out + (size_t)row * P.ld_out + t.n0 + c;
 #pragma unroll
-            for (int v = 0; v < 8; ++v)
-              if (c + 4 * v < ncols)
-                *reinterpret_cast<uint4*>(out + 4 * v) = make_uint4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
-          } else {
-            __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + n0 + c;
+              for (int v = 0; v < 8; ++v)
+                if (c + 4 * v < ncols)
+                  *reinterpret_cast<uint4*>(out + 4 * v) = make_uint4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
+            } else {
+              __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + t.n0 + c;
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (c + 8 * v < ncols) {
-                uint32_t o[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                  o[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]), __uint_as_float(a[8 * v + 2 * j + 1]));
-                *reinterpret_cast<uint4*>(out + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
-                if (P.split) {
-                  uint32_t ol[4];
+              for (int v = 0; v < 4; ++v) {
+                if (c + 8 * v < ncols) {
+                  uint32_t o[4];
 #pragma unroll
                   for (int j = 0; j < 4; ++j)
-                    ol[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
-                                        __uint_as_float(a[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
-                  *reinterpret_cast<uint4*>(out + P.out_off_lo + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                    o[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]), __uint_as_float(a[8 * v + 2 * j + 1]));
+                  *reinterpret_cast<uint4*>(out + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
+                  if (P.split) {
+                    uint32_t ol[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                      ol[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
+                                          __uint_as_float(a[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
+                    *reinterpret_cast<uint4*>(out + P.out_off_lo + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                  }
                 }
               }
             }
           }
         }
       }
-     }
-    } else if (lane == 0) {
-      flag_error(P.st, MOE_ERR_TIMEOUT, 0x402u);
+      // the accumulators are in registers / memory now: hand TMEM back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.accum_empty);
     }
   }
   // ---- teardown: every role gets here in bounded time
@@ -435,12 +474,15 @@ int launch_gg(moe_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const 
   const size_t stage_bytes = (size_t)kBM * kBK * 2 * 2 + 256 * kBK * 2;
   const size_t smem = P.n_stages * stage_bytes + sizeof(SmemGG) + 1024 + 128;
   if ((long long)smem > ctx->max_smem_optin) return MOE_ERR_UNSUPPORTED;
-  const int tile_rows = P.dual_a ? kBM : kTileRows;
-  const int m_tiles = (n_slots + tile_rows - 1) / tile_rows + c.n_experts;  // upper bound over all groupings
   const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
-  if (m_tiles > 65535) return MOE_ERR_UNSUPPORTED;
+  // 256-row tiles halve the operand traffic per flop; small problems keep 128-row tiles to fill the SMs
+  P.tile_rows = kBM;
+  if (!P.dual_a && (long long)((n_slots + kTileRows - 1) / kTileRows) * n_tiles >= 2ll * ctx->sm_count)
+    P.tile_rows = kTileRows;
+  const long long m_tiles = (n_slots + P.tile_rows - 1) / P.tile_rows + c.n_experts;  // upper bound
+  const int grid = (int)std::min<long long>(m_tiles * n_tiles, ctx->sm_count);
   MOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  grouped_gemm_kernel<<<dim3(n_tiles, m_tiles), kThreadsGG, smem, s>>>(a0, a1, b, P);
+  grouped_gemm_kernel<<<grid, kThreadsGG, smem, s>>>(a0, a1, b, P);
   MOE_CUDA_TRY(cudaGetLastError());
   ctx->launches++;
   return MOE_OK;
