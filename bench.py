@@ -154,7 +154,7 @@ def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use
     # CUDA graph of one trip around the ring (decode steps are launch-bound otherwise)
     graph = None
     mode = "stream"
-    if kind == "decode" and use_graph:
+    if use_graph:
         try:
             g = torch.cuda.CUDAGraph()
             side = torch.cuda.Stream()

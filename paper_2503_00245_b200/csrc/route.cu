@@ -23,31 +23,45 @@ __device__ __forceinline__ void load_x8<__nv_bfloat16>(const __nv_bfloat16* p, f
 
 constexpr int kRouteWarps = 8;
 
-// Partial logits of one token over the chunks [c_begin, c_end) step c_step of the d axis.
+// Partial logits of one token over the chunks [c_begin, c_end) step c_step of the d axis.  The token's
+// chunks are fetched eight at a time before any arithmetic, so a warp pays one memory round trip per group.
 template <typename XT, int EMAX>
 __device__ __forceinline__ void route_partial(const XT* __restrict__ xr, const uint16_t* __restrict__ w_router, int E,
                                               int c_begin, int c_end, int c_step, float* acc) {
   const bool vec = (E % 8) == 0;
-  for (int c = c_begin; c < c_end; c += c_step) {
-    float xv[8];
-    load_x8<XT>(xr + c * 8, xv);
+  for (int cb = c_begin; cb < c_end; cb += 8 * c_step) {
+    float xv[8][8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const uint16_t* wr = w_router + (size_t)(c * 8 + i) * E;
-      if (vec) {
-#pragma unroll
-        for (int e8 = 0; e8 < EMAX / 8; ++e8) {
-          if (e8 * 8 < E) {
-            float wv[8];
-            unpack8(__ldg(reinterpret_cast<const uint4*>(wr) + e8), wv);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) acc[e8 * 8 + j] = fmaf(xv[i], wv[j], acc[e8 * 8 + j]);
-          }
-        }
+    for (int u = 0; u < 8; ++u) {
+      const int c = cb + u * c_step;
+      if (c < c_end) {
+        load_x8<XT>(xr + c * 8, xv[u]);
       } else {
 #pragma unroll
-        for (int e = 0; e < EMAX; ++e)
-          if (e < E) acc[e] = fmaf(xv[i], bf16_to_float(__ldg(wr + e)), acc[e]);
+        for (int i = 0; i < 8; ++i) xv[u][i] = 0.f;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int c = min(cb + u * c_step, c_end - 1);  // clamped rows meet zero inputs
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint16_t* wr = w_router + (size_t)(c * 8 + i) * E;
+        if (vec) {
+#pragma unroll
+          for (int e8 = 0; e8 < EMAX / 8; ++e8) {
+            if (e8 * 8 < E) {
+              float wv[8];
+              unpack8(__ldg(reinterpret_cast<const uint4*>(wr) + e8), wv);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) acc[e8 * 8 + j] = fmaf(xv[u][i], wv[j], acc[e8 * 8 + j]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < EMAX; ++e)
+            if (e < E) acc[e] = fmaf(xv[u][i], bf16_to_float(__ldg(wr + e)), acc[e]);
+        }
       }
     }
   }
