@@ -309,12 +309,108 @@ def cpu_baseline(name, budget_s=12.0):
             "sample": f"{n} forward passes of layer 0 of the ring ({el:.1f} s of CPU time), numpy fp64"}
 
 
+def run_offload_stack(a, device):
+    """Stacked decode with host-resident experts: n_layers phone-scale layers (E = 16, top-2), `slots` experts
+    per layer resident in HBM, the rest in pinned host memory, Zipf(1.2)-skewed routing; one step = one token
+    through all layers.  Reports us/token and the host-link traffic against the measured pinned H2D rate."""
+    import paper_2503_00245_b200 as P
+    from paper_2503_00245_b200 import binding as B
+    sh = W.PHONE_OFFLOAD
+    n_layers, slots, steps = a.layers, a.slots, a.decode_steps
+    layers = []
+    for l in range(n_layers):
+        r_w, r_b = W.make_router(sh, device, l)
+        ex = W.make_experts(sh, device, l)
+        layers.append({"w_router": r_w, "b_router": r_b, "gud": P.pack_dense(ex["w_gate"], ex["w_up"], ex["w_down"])})
+        del ex
+        if l % 4 == 3:
+            torch.cuda.synchronize()
+    def gen():
+        for lay in layers:
+            yield lay
+            lay["gud"] = None          # the device copy is no longer needed once it is in pinned memory
+    stack = P.OffloadedStack(sh.d_model, sh.d_ff, sh.n_experts, sh.top_k, slots, gen())
+    torch.cuda.empty_cache()
+    # pinned host->device bandwidth of this box (the roofline of a miss)
+    probe_dst = torch.empty(stack.slot_bytes, dtype=torch.uint8, device=device)
+    src = stack.host[0].view(torch.uint8).reshape(-1)[:stack.slot_bytes]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    probe_dst.copy_(src, non_blocking=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(8):
+        probe_dst.copy_(src, non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    h2d_gbs = 8 * stack.slot_bytes / (e0.elapsed_time(e1) * 1e-3) / 1e9
+    hs = [W.make_x(sh.with_(x_dtype="f32"), 1, device=device, step=s)[0].contiguous() for s in range(steps + 3)]
+    for s in range(3):
+        stack.step(hs[steps + s].clone())
+    torch.cuda.synchronize()
+    st0 = stack.stats()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    trace = []
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0.record()
+    for s in range(steps):
+        trace.append(stack.step(hs[s]))
+    e1.record()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    clocks = sampler.stop()
+    assert stack.check() == 0
+    ms = e0.elapsed_time(e1)
+    st1 = stack.stats()
+    fetches, nbytes, hits = (st1[k] - st0[k] for k in ("fetches", "bytes", "hits"))
+    lookups = steps * n_layers * sh.top_k
+    # Eq. 4-5 on the routing the layers produced, per layer (B = layers, T = steps)
+    tr = torch.tensor(trace, dtype=torch.int32, device=device).permute(1, 0, 2).contiguous()
+    hsum = torch.zeros(1, dtype=torch.int64, device=device)
+    B.moe_expert_replacements(tr, n_layers, steps, sh.top_k, sh.n_experts, hsum)
+    torch.cuda.synchronize()
+    exrep = (int(hsum.item()) // 2) / (n_layers * sh.top_k * max(1, steps - 1))
+    us_tok = ms * 1e3 / steps
+    bytes_tok = nbytes / steps
+    t_link = bytes_tok / (h2d_gbs * 1e9) * 1e6
+    t_hbm = n_layers * sh.top_k * W.expert_bytes(sh) / (peaks()["hbm_gbs"] * 1e9) * 1e6
+    line = {
+        "metric": "moe_stack_us_per_token_decode_offload", "value": round(us_tok, 2), "unit": "us/token",
+        "n_gpus": 1, "steps": steps, "warmup": 3, "ms_per_step": round(ms / steps, 4), "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/activations, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": "phone-offload-stack", "shape": W.describe(sh), "layers": n_layers,
+                   "resident_slots_per_layer": slots, "T": 1, "launch_mode": "stream (host sync per layer)",
+                   "l2": "inputs larger than L2: 24 distinct layers per token"},
+        "roofline": {"bound": "host_link", "achieved": round(bytes_tok / (us_tok * 1e-6) / 1e9, 2),
+                     "peak": round(h2d_gbs, 2), "unit": "GB/s",
+                     "frac": round(t_link / us_tok, 4), "traffic": None,
+                     "peak_source": "pinned H2D copy of one expert, measured in this run",
+                     "note": "frac = (fetch bytes / measured H2D rate) / time per token"},
+        "offload": {"fetch_bytes_per_token": int(bytes_tok), "fetches_per_token": round(fetches / steps, 3),
+                    "hit_rate": round(hits / lookups, 4), "exrep": round(exrep, 4),
+                    "no_miss_floor_us": round(t_hbm, 1), "host_link_floor_us": round(t_link, 1),
+                    "host_wall_us_per_token": round(wall * 1e6 / steps, 1)},
+        "e2e": {"value": round(wall * 1e6 / steps, 2), "unit": "us/token", "h2d_bytes_per_step": int(bytes_tok),
+                "d2h_bytes_per_step": n_layers * sh.top_k * 4},
+        "gpu_launches": int(B.moe_launch_count(stack.ctx)),
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    stack.close()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4096)
     ap.add_argument("--warmup", type=int, default=64)
-    ap.add_argument("--workload", default=DEFAULT, choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT, choices=sorted(WORKLOADS) + ["phone-offload-stack"])
+    ap.add_argument("--layers", type=int, default=24, help="phone-offload-stack: stacked layers")
+    ap.add_argument("--slots", type=int, default=4, help="phone-offload-stack: resident experts per layer")
+    ap.add_argument("--decode-steps", type=int, default=256, help="phone-offload-stack: tokens")
     ap.add_argument("--all", action="store_true", help="also time the other workloads (reported under 'others')")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -354,6 +450,8 @@ def main():
     if world > 1:
         torch.distributed.barrier()
 
+    if a.workload == "phone-offload-stack":
+        return run_offload_stack(a, device) if rank == 0 else 0
     res = time_workload(a.workload, a.steps, a.warmup, device, rank, world, a.ring, not a.no_graph)
     ms_tot = torch.tensor([res["ms_total"]], device=device, dtype=torch.float64)
     if world > 1:
