@@ -56,6 +56,8 @@ struct DenseParams {
   DeviceState* st;
   long long* acc;
   int stage_bytes, n_stages, xs_bytes;
+  int acc_copies;              // the CTAs spread their atomics over this many accumulator copies
+  long long acc_copy_stride;   // elements between copies
 };
 
 struct Smem {
@@ -309,7 +311,8 @@ __device__ __forceinline__ bool consume_pass(const DenseParams& P, Smem& sm, con
       if (s < n) {
         const int gs = slot0 + s;
         const int rowi = P.mode == 0 ? sm.slot_tok[gs] : gs;
-        unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) + (size_t)rowi * d + mychunk * 8;
+        unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) +
+                                  (size_t)(blockIdx.x % P.acc_copies) * P.acc_copy_stride + (size_t)rowi * d + mychunk * 8;
 #pragma unroll
         for (int j = 0; j < 8; ++j) atomicAdd(dst + j, (unsigned long long)__float2ll_rn(acc[s][j] * kFixScale));
       }
@@ -342,6 +345,12 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     fence_proxy_async_smem();
     sm.abort = 0;
     sm.last = 0;
+    if (P.fused_route) {
+      // one token: every pass reads token row 0, so the first pass's copy of x can start before the routing
+      const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
+      mbar_arrive_expect_tx(&sm.xfull[0], xrow_bytes);
+      bulk_g2s(xs, P.x, xrow_bytes, &sm.xfull[0]);
+    }
   }
   if (P.fused_route) {
     // router logits of the single token: every consumer thread takes rows of W_r (row i = the E weights
@@ -390,22 +399,40 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
       }
     }
+    float bias0 = 0.f, bias1 = 0.f;
+    if (warp == 0 && P.b_router) {  // fetched while the logits are being reduced
+      if (lane < P.E) bias0 = P.b_router[lane];
+      if (lane + 32 < P.E) bias1 = P.b_router[lane + 32];
+    }
     __syncthreads();
     if (warp == 0) {
-      float l0 = 0.f, l1 = 0.f;
-      if (lane < P.E) {
+      float l0 = bias0, l1 = bias1;
+      if (lane < P.E)
         for (int w = 0; w < kWarps; ++w) l0 += sm.red[w][lane];
-        if (P.b_router) l0 += P.b_router[lane];
-      }
-      if (lane + 32 < P.E) {
+      if (lane + 32 < P.E)
         for (int w = 0; w < kWarps; ++w) l1 += sm.red[w][lane + 32];
-        if (P.b_router) l1 += P.b_router[lane + 32];
-      }
       warp_route_finish(l0, l1, P.E, P.k, P.renorm, lane, sm.stage_e, sm.stage_w, nullptr);
       __syncwarp();
-      if (blockIdx.x == 0 && lane < P.k) {
-        if (P.topk_idx) P.topk_idx[lane] = sm.stage_e[lane];
-        if (P.topk_w) P.topk_w[lane] = sm.stage_w[lane];
+      // the k selected experts in ascending order are the active experts, one slot (token 0) each
+      if (lane < P.k) {
+        const int e = sm.stage_e[lane];
+        int rank = 0;
+        for (int i = 0; i < P.k; ++i) rank += (sm.stage_e[i] < e);
+        const int sl = P.expert_slot ? P.expert_slot[e] : e;
+        if (sl < 0) flag_error(st, MOE_ERR_STATE, 0x301u);
+        sm.act_e[rank] = e;
+        sm.act_slot[rank] = sl < 0 ? 0 : sl;
+        sm.act_off[rank] = rank;
+        sm.slot_tok[rank] = 0;
+        sm.slot_w[rank] = sm.stage_w[lane];
+        if (blockIdx.x == 0) {
+          if (P.topk_idx) P.topk_idx[lane] = e;
+          if (P.topk_w) P.topk_w[lane] = sm.stage_w[lane];
+        }
+      }
+      if (lane == 0) {
+        sm.act_off[P.k] = P.k;
+        sm.n_act = P.k;
       }
     }
   } else if (P.mode == 0 && warp == 0) {
@@ -415,7 +442,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     }
   }
   __syncthreads();
-  if (tid == 0) {
+  if (tid == 0 && !P.fused_route) {
     // routing products -> active experts and their slots (same numbering as moe_permute)
     const int n = n_pairs;
     int na = 0, bad = 0;
@@ -511,14 +538,16 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
         known_free = L;
       }
-      // the pass's token rows
+      // the pass's token rows (pass 0 of a single-token launch: already on its way since the prologue)
       const int slot0 = sm.act_off[ps.ai] + ps.s0;
-      fence_proxy_async_smem();
       ++pn_issued;
-      mbar_arrive_expect_tx(&sm.xfull[b], (uint32_t)ps.ns * xrow_bytes);
-      for (int s = 0; s < ps.ns; ++s)
-        bulk_g2s(xs + (size_t)b * P.xs_bytes + (size_t)s * xrow_bytes,
-                 (const unsigned char*)P.x + (size_t)sm.slot_tok[slot0 + s] * xrow_bytes, xrow_bytes, &sm.xfull[b]);
+      if (!(P.fused_route && pn == 0)) {
+        fence_proxy_async_smem();
+        mbar_arrive_expect_tx(&sm.xfull[b], (uint32_t)ps.ns * xrow_bytes);
+        for (int s = 0; s < ps.ns; ++s)
+          bulk_g2s(xs + (size_t)b * P.xs_bytes + (size_t)s * xrow_bytes,
+                   (const unsigned char*)P.x + (size_t)sm.slot_tok[slot0 + s] * xrow_bytes, xrow_bytes, &sm.xfull[b]);
+      }
       const unsigned char* src = reinterpret_cast<const unsigned char*>(P.gud) +
                                  ((size_t)sm.act_slot[ps.ai] * P.f + ps.ra) * row_bytes;
       for (int row = ps.ra; row < ps.rb; row += kRows) {
@@ -545,6 +574,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       last_idx[b] = rp.n - 1;
       ++pn;
     }
+    if (P.fused_route && pn_issued == 0) (void)mbar_wait(&sm.xfull[0], 0u);  // the early copy of x must land
     if (!ok) {
       // copies already in flight must land before this CTA's shared memory goes away
       for (int back = 1; back <= NS && back <= rp.n; ++back) {
@@ -597,8 +627,12 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     const long long total = (long long)rows * P.d;
     const bool good = ld_acquire(&st->status) == 0u;
     for (long long i = tid; i < total; i += kConsumerThreads) {
-      const long long v = __ldcg(P.acc + i);
-      P.acc[i] = 0;
+      long long v = 0;
+      for (int c = 0; c < P.acc_copies; ++c) {
+        long long* p = P.acc + (size_t)c * P.acc_copy_stride + i;
+        v += __ldcg(p);
+        *p = 0;
+      }
       if (!good) continue;
       const float fv = (float)((double)v * kFixInv);
       if (P.mode == 1)
@@ -629,6 +663,14 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   P.topk_idx = topk_idx, P.topk_w = topk_w, P.offsets = offsets, P.perm = perm;
   P.expert_slot = w->expert_slot, P.gud = (const uint16_t*)w->gud;
   P.y = y, P.out_slots = out_slots, P.st = ctx->d_state, P.acc = ctx->acc;
+  {
+    // contended atomics on few lines are slow: with room in the accumulator buffer, CTAs use up to 8 copies
+    const long long rows = (mode == 0) ? T : (long long)T * c.top_k;
+    P.acc_copy_stride = rows * c.d_model;
+    const long long fit = (long long)ctx->acc_elems / P.acc_copy_stride;
+    if (fit < 1) return MOE_ERR_UNSUPPORTED;
+    P.acc_copies = (int)(fit < 8 ? fit : 8);
+  }
   const int xrow = c.d_model * (P.x_is_bf16 ? 2 : 4);
   P.xs_bytes = (min(T, kMaxN) * xrow + 127) / 128 * 128;
   P.stage_bytes = kRows * 3 * c.d_model * 2;  // multiple of 16; the ring base is 128-byte aligned
@@ -727,7 +769,7 @@ extern "C" int moe_layer_forward_static(const moe_config* cfg, const void* x, in
   // The array keeps what the last call left.  A call that ran to its end leaves the accumulators and the
   // arrival counter at zero, one that was cut short does not: clear the part this call uses, keep the status.
   MOE_CUDA_TRY(cudaMemsetAsync(&st->done_count, 0, sizeof(unsigned int), s));
-  MOE_CUDA_TRY(cudaMemsetAsync(acc, 0, (size_t)T * cfg->d_model * sizeof(long long), s));
+  MOE_CUDA_TRY(cudaMemsetAsync(acc, 0, kStaticAccBytes, s));
   moe_ctx tmp{};  // a view, not a context: nothing here owns memory
   tmp.cfg = *cfg;
   tmp.cfg.path = MOE_PATH_STREAM;
