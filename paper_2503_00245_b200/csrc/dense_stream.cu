@@ -626,21 +626,36 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     const int rows = P.mode == 0 ? P.T : n_pairs;
     const long long total = (long long)rows * P.d;
     const bool good = ld_acquire(&st->status) == 0u;
-    for (long long i = tid; i < total; i += kConsumerThreads) {
-      long long v = 0;
-      for (int c = 0; c < P.acc_copies; ++c) {
-        long long* p = P.acc + (size_t)c * P.acc_copy_stride + i;
-        v += __ldcg(p);
-        *p = 0;
+    // four outputs per thread at a time: all their copies are fetched in one round trip, then summed,
+    // converted, stored, and the copies zeroed
+    for (long long i0 = tid; i0 < total; i0 += 4 * kConsumerThreads) {
+      long long part[4][8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const long long i = i0 + (long long)j * kConsumerThreads;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          part[j][c] = (i < total && c < P.acc_copies) ? __ldcg(P.acc + (size_t)c * P.acc_copy_stride + i) : 0ll;
       }
-      if (!good) continue;
-      const float fv = (float)((double)v * kFixInv);
-      if (P.mode == 1)
-        P.out_slots[i] = fv;
-      else if (P.x_is_bf16)
-        ((__nv_bfloat16*)P.y)[i] = __float2bfloat16_rn(fv);
-      else
-        ((float*)P.y)[i] = fv;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const long long i = i0 + (long long)j * kConsumerThreads;
+        if (i >= total) continue;
+        long long v = 0;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          v += part[j][c];
+          if (c < P.acc_copies) P.acc[(size_t)c * P.acc_copy_stride + i] = 0;
+        }
+        if (!good) continue;
+        const float fv = (float)((double)v * kFixInv);
+        if (P.mode == 1)
+          P.out_slots[i] = fv;
+        else if (P.x_is_bf16)
+          ((__nv_bfloat16*)P.y)[i] = __float2bfloat16_rn(fv);
+        else
+          ((float*)P.y)[i] = fv;
+      }
     }
     if (tid == 0) st->done_count = 0u;
   }
