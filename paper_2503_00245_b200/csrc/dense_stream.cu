@@ -56,6 +56,7 @@ struct DenseParams {
   DeviceState* st;
   long long* acc;
   int stage_bytes, n_stages, xs_bytes;
+  int wpart_ok;                // shared memory holds the [8][d] merge buffer of the unit-owner passes (d <= 1024)
   int acc_copies;              // the CTAs spread their atomics over this many accumulator copies
   long long acc_copy_stride;   // elements between copies
 };
@@ -184,6 +185,102 @@ __device__ __forceinline__ bool consumer_sync(Smem& sm, unsigned& par, int lane)
   const bool ok = mbar_wait_spin(&sm.cbar, par);
   par ^= 1u;
   return ok;
+}
+
+// One pass with a single token and d <= 1024: warp (g, r) = (warp >> 2, warp & 3) owns hidden unit r of the
+// stages whose ring index has parity g, and does all of that unit's work -- both dot products, h, and the
+// update of a d-wide partial output it keeps in registers (lane owns chunks lane, lane + 32, ...) -- so
+// warps never wait for each other inside the pass.  At the end the eight partial outputs are summed in a
+// fixed order through shared memory and leave as fixed-point atomics.
+constexpr int kT1Iters = 4;  // 16-byte chunks of a row per lane
+__device__ __forceinline__ bool consume_pass_t1(const DenseParams& P, Smem& sm, const Pass& ps, const unsigned char* ring,
+                                                const unsigned char* xs, float* wpart, RingPos& rp, unsigned& cpar,
+                                                int warp, int lane) {
+  DeviceState* st = P.st;
+  const int NS = P.n_stages, d = P.d, chunks = d >> 3, cl = chunks - 1;
+  const bool xbf = P.x_is_bf16 != 0;
+  const int slot0 = sm.act_off[ps.ai] + ps.s0;
+  const float wgt = sm.slot_w[slot0];
+  const int grp = warp >> 2, r = warp & 3;
+  float4 xr[kT1Iters][2];
+  float acc[kT1Iters][8];
+  int cidx[kT1Iters];
+#pragma unroll
+  for (int it = 0; it < kT1Iters; ++it) {
+    const int c = lane + 32 * it;
+    cidx[it] = min(c, cl);
+    load_x_chunk(xs, cidx[it], xbf, xr[it][0], xr[it][1]);
+    if (c > cl) xr[it][0] = xr[it][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[it][j] = 0.f;
+  }
+  for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
+    const int nrows = min(kRows, ps.rb - row0);
+    if (!mbar_wait(&sm.full[rp.slot], rp.par)) {
+      if (lane == 0) set_abort(st, sm, 0x313u);
+      return false;
+    }
+    if ((rp.n & 1) == grp && r < nrows) {
+      const uint4* base = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * P.stage_bytes) + (size_t)r * 3 * chunks;
+      uint4 wg[kT1Iters], wu[kT1Iters], wd[kT1Iters];
+#pragma unroll
+      for (int it = 0; it < kT1Iters; ++it) wg[it] = base[cidx[it]];
+#pragma unroll
+      for (int it = 0; it < kT1Iters; ++it) wu[it] = base[chunks + cidx[it]];
+#pragma unroll
+      for (int it = 0; it < kT1Iters; ++it) wd[it] = base[2 * chunks + cidx[it]];
+      float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;
+#pragma unroll
+      for (int it = 0; it < kT1Iters; ++it) {
+        dot8(wg[it], xr[it][0], xr[it][1], g0, g1);
+        dot8(wu[it], xr[it][0], xr[it][1], u0, u1);
+      }
+      float g = g0 + g1, u = u0 + u1;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        g += __shfl_xor_sync(0xffffffffu, g, o);
+        u += __shfl_xor_sync(0xffffffffu, u, o);
+      }
+      const float h = g / (1.0f + expf(-g)) * u * wgt;
+#pragma unroll
+      for (int it = 0; it < kT1Iters; ++it) {
+        float w[8];
+        unpack8(wd[it], w);
+        const float hh = (lane + 32 * it <= cl) ? h : 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[it][j] = fmaf(hh, w[j], acc[it][j]);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) {
+      mbar_arrive(&sm.hbar[rp.slot]);  // keeps this barrier's phase in step with the slot's uses
+      mbar_arrive(&sm.freeb[rp.slot]);
+    }
+    rp.advance(NS);
+  }
+  // ---- sum the eight warps' partial outputs in a fixed order, send the CTA's sum to the global accumulators
+  float* mine = wpart + (size_t)warp * d;
+#pragma unroll
+  for (int it = 0; it < kT1Iters; ++it) {
+    if (lane + 32 * it <= cl) {
+      float4* q = reinterpret_cast<float4*>(mine + (lane + 32 * it) * 8);
+      q[0] = make_float4(acc[it][0], acc[it][1], acc[it][2], acc[it][3]);
+      q[1] = make_float4(acc[it][4], acc[it][5], acc[it][6], acc[it][7]);
+    }
+  }
+  if (!consumer_sync(sm, cpar, lane)) return false;
+  {
+    const int rowi = P.mode == 0 ? sm.slot_tok[slot0] : slot0;
+    unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) +
+                              (size_t)(blockIdx.x % P.acc_copies) * P.acc_copy_stride + (size_t)rowi * d;
+    for (int i = warp * 32 + lane; i < d; i += kConsumerThreads) {
+      float v = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) v += wpart[(size_t)w * d + i];
+      atomicAdd(dst + i, (unsigned long long)__float2ll_rn(v * kFixScale));
+    }
+  }
+  return consumer_sync(sm, cpar, lane);  // wpart may be rewritten by the next pass
 }
 
 // One pass of the consumers: units [ra, rb) of one expert for NT tokens (NT == 1: the token row lives
@@ -326,6 +423,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   unsigned char* ring = smem_raw + kSmemHeaderBytes;
   unsigned char* xs = ring + (size_t)P.n_stages * P.stage_bytes;  // 2 buffers of xs_bytes
+  float* wpart = reinterpret_cast<float*>(xs + 2 * (size_t)P.xs_bytes);  // [8 warps][d], single-token passes at d <= 1024
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NS = P.n_stages;
   DeviceState* const st = P.st;
@@ -587,6 +685,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   }
 
   // ===================================================================== consumers
+  unsigned cpar = 0;
   {
     bool ok = true;
     int pn = 0;
@@ -598,7 +697,9 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         break;
       }
       const unsigned char* xsb = xs + (size_t)b * P.xs_bytes;
-      if (ps.ns == 1)
+      if (ps.ns == 1 && P.wpart_ok)
+        ok = consume_pass_t1(P, sm, ps, ring, xsb, wpart, rp, cpar, warp, lane);
+      else if (ps.ns == 1)
         ok = consume_pass<1>(P, sm, ps, ring, xsb, rp, warp, lane);
       else if (ps.ns == 2)
         ok = consume_pass<2>(P, sm, ps, ring, xsb, rp, warp, lane);
@@ -612,7 +713,6 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   // ------------------------------------------------------------------ all partial sums are out
   // (after an expired wait the warps may be out of step with this barrier: then it can expire too; the
   // status word is already set and nobody finalises)
-  unsigned cpar = 0;
   bool fin = consumer_sync(sm, cpar, lane);
   if (tid == 0) {
     __threadfence();
@@ -690,7 +790,8 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   P.xs_bytes = (min(T, kMaxN) * xrow + 127) / 128 * 128;
   P.stage_bytes = kRows * 3 * c.d_model * 2;  // multiple of 16; the ring base is 128-byte aligned
   P.stage_bytes = (P.stage_bytes + 127) / 128 * 128;
-  const size_t fixed = 2 * (size_t)P.xs_bytes + kSmemHeaderBytes + 256;
+  P.wpart_ok = c.d_model <= 32 * 8 * kT1Iters ? 1 : 0;
+  const size_t fixed = 2 * (size_t)P.xs_bytes + (P.wpart_ok ? (size_t)kWarps * c.d_model * 4 : 0) + kSmemHeaderBytes + 256;
   const long long avail = (long long)ctx->max_smem_optin - (long long)fixed;
   if (avail < 2ll * P.stage_bytes) return MOE_ERR_UNSUPPORTED;
   P.n_stages = (int)min((long long)kMaxStages, avail / P.stage_bytes);
