@@ -430,6 +430,10 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   const int n_pairs = P.T * P.k;
 
   // ------------------------------------------------------------------ prologue
+  // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as this one's CTAs
+  // leave their SMs (its set-up then overlaps this kernel's last CTAs); this kernel in turn reads nothing a
+  // predecessor may have written (x, routing, accumulators) before griddepcontrol.wait below.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == kConsumerThreads) {  // the producer thread sets up the barriers
     for (int i = 0; i < NS; ++i) {
       mbar_init(&sm.full[i], 1);
@@ -443,6 +447,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     fence_proxy_async_smem();
     sm.abort = 0;
     sm.last = 0;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (P.fused_route) {
       // one token: every pass reads token row 0, so the first pass's copy of x can start before the routing
       const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
@@ -450,6 +455,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       bulk_g2s(xs, P.x, xrow_bytes, &sm.xfull[0]);
     }
   }
+  if (tid != kConsumerThreads) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (P.fused_route) {
     // router logits of the single token: every consumer thread takes rows of W_r (row i = the E weights
     // of input feature i), 8 experts at a time
@@ -798,8 +804,13 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   const size_t smem = (size_t)P.n_stages * P.stage_bytes + fixed;
   const int G = ctx->sm_count;
   MOE_CUDA_TRY(cudaFuncSetAttribute(dense_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  dense_stream_kernel<<<G, kThreads, smem, s>>>(P);
-  MOE_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3(G), lc.blockDim = dim3(kThreads), lc.dynamicSmemBytes = smem, lc.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr, lc.numAttrs = 1;
+  MOE_CUDA_TRY(cudaLaunchKernelEx(&lc, dense_stream_kernel, P));
   ctx->launches++;
   return MOE_OK;
 }
