@@ -455,6 +455,15 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       bulk_g2s(xs, P.x, xrow_bytes, &sm.xfull[0]);
     }
   }
+  // the router's weights do not depend on any earlier kernel: the first group of eight experts is fetched
+  // before the dependency wait, so its DRAM latency overlaps the predecessor's tail
+  uint4 wr0[kXIters];
+  const bool prefetched = P.fused_route && warp < kWarps && (P.E & 7) == 0;
+  if (prefetched) {
+#pragma unroll
+    for (int j = 0; j < kXIters; ++j)
+      wr0[j] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + j * kConsumerThreads, P.d - 1) * P.E));
+  }
   if (tid != kConsumerThreads) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (P.fused_route) {
     // router logits of the single token: every consumer thread takes rows of W_r (row i = the E weights
@@ -474,7 +483,9 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           uint4 wr[kXIters];
 #pragma unroll
           for (int j = 0; j < kXIters; ++j)
-            wr[j] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + j * kConsumerThreads, d - 1) * E + e8));
+            wr[j] = e8 == 0 ? wr0[j]
+                            : __ldg(reinterpret_cast<const uint4*>(P.w_router +
+                                                                   (size_t)min(tid + j * kConsumerThreads, d - 1) * E + e8));
           float a[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) a[j] = 0.f;
