@@ -228,7 +228,7 @@ def roofline(res):
         ach = b / sec / 1e9
         return {"bound": "hbm", "achieved": round(ach, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": round(ach / pk["hbm_gbs"], 4), "traffic": None, "peak_source": pk["source"],
-                "bytes_per_launch": int(b), "kernel": "stream_ffn_kernel",
+                "bytes_per_launch": int(b), "kernel": "dense_stream_kernel",
                 "note": "duration = whole step (router + expert kernel) / 1"}
     fl = flops(shape, T)
     t_tc = fl / (pk["tflops_sustained"] * 1e12)
@@ -402,6 +402,20 @@ def run_offload_stack(a, device):
     return 0
 
 
+def max_over_ranks(value: float, world: int, device="cpu") -> float:
+    """A time measured on every rank -> the slowest rank's (all ranks get it).  Replicas exchange nothing else."""
+    if world <= 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate(metric_kind: str, T: int, ms_per_step: float, world: int):
+    """Whole-job value for `world` replicas that each ran the same steps in ms_per_step (max over ranks)."""
+    return metric_of({"T": T, "kind": metric_kind}, ms_per_step, world)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -453,16 +467,10 @@ def main():
     if a.workload == "phone-offload-stack":
         return run_offload_stack(a, device) if rank == 0 else 0
     res = time_workload(a.workload, a.steps, a.warmup, device, rank, world, a.ring, not a.no_graph)
-    ms_tot = torch.tensor([res["ms_total"]], device=device, dtype=torch.float64)
-    if world > 1:
-        torch.distributed.all_reduce(ms_tot, op=torch.distributed.ReduceOp.MAX)
-    ms_per_step = float(ms_tot.item()) / res["steps"]
+    ms_per_step = max_over_ranks(res["ms_total"], world, device) / res["steps"]
     metric, value, unit, hib = metric_of(res, ms_per_step, world)
     e2e_ms, h2d, d2h = e2e_measure(res, a.steps)
-    e2e_t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
-    if world > 1:
-        torch.distributed.all_reduce(e2e_t, op=torch.distributed.ReduceOp.MAX)
-    _, e2e_val, _, _ = metric_of(res, float(e2e_t.item()), world)
+    _, e2e_val, _, _ = metric_of(res, max_over_ranks(e2e_ms, world, device), world)
 
     others = []
     if a.all and rank == 0 and world == 1:
