@@ -56,6 +56,8 @@ struct DenseParams {
   DeviceState* st;
   long long* acc;
   int stage_bytes, n_stages, xs_bytes;
+  int unit_stride;             // bytes between the hidden units of a stage (3 rows, padded for the MMA passes)
+  int use_mma;                 // more than one token: every pass goes through consume_pass_mma
   int wpart_ok;                // shared memory holds the [8][d] merge buffer of the unit-owner passes (d <= 1024)
   int acc_copies;              // the CTAs spread their atomics over this many accumulator copies
   long long acc_copy_stride;   // elements between copies
@@ -67,8 +69,10 @@ struct Smem {
   uint64_t freeb[kMaxStages];  // all consumer warps are done with the stage
   uint64_t xfull[2];           // token rows of a pass landed in xs[0/1]
   uint64_t cbar;               // barrier over the consumer warps
-  float gu[kMaxStages][kRows * 2][kMaxN];
-  float red[kWarps][MOE_MAX_EXPERTS];
+  float gu[kMaxStages][kRows * 2];     // single-token passes at d > 1024: the stage's 8 dot products
+  __align__(16) float red[2][2][kWarps][kRows * 8];  // multi-token passes: [stage parity][gate | up][warp][unit * 8 + token]
+  __align__(16) uint32_t zero16[4];    // what ldmatrix reads for padding rows
+  float rlog[kWarps][MOE_MAX_EXPERTS];
   int act_e[MOE_MAX_EXPERTS];
   int act_slot[MOE_MAX_EXPERTS];
   int act_off[MOE_MAX_EXPERTS + 1];
@@ -221,7 +225,7 @@ __device__ __forceinline__ bool consume_pass_t1(const DenseParams& P, Smem& sm, 
       return false;
     }
     if ((rp.n & 1) == grp && r < nrows) {
-      const uint4* base = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * P.stage_bytes) + (size_t)r * 3 * chunks;
+      const uint4* base = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * P.stage_bytes + (size_t)r * P.unit_stride);
       uint4 wg[kT1Iters], wu[kT1Iters], wd[kT1Iters];
 #pragma unroll
       for (int it = 0; it < kT1Iters; ++it) wg[it] = base[cidx[it]];
@@ -283,117 +287,165 @@ __device__ __forceinline__ bool consume_pass_t1(const DenseParams& P, Smem& sm, 
   return consumer_sync(sm, cpar, lane);  // wpart may be rewritten by the next pass
 }
 
-// One pass of the consumers: units [ra, rb) of one expert for NT tokens (NT == 1: the token row lives
-// in registers; otherwise the rows are read from shared memory for every dot product).
-template <int NT>
-__device__ __forceinline__ bool consume_pass(const DenseParams& P, Smem& sm, const Pass& ps, const unsigned char* ring,
-                                             const unsigned char* xs, RingPos& rp, int warp, int lane) {
+// ---------------------------------------------------------------------------------------------------
+// Passes with several tokens: the same streamed bytes, but the per-token arithmetic goes to the tensor cores
+// (mma.sync m16n8k16, bf16 inputs, fp32 accumulation) so that the instruction count does not grow with the
+// number of tokens and the path stays bound by the weight stream.  Up to 8 tokens per pass (the MMA's N).
+//
+// Per stage of 4 hidden units:
+//  (1) gate/up logits: D[8 weight rows][8 tokens] = W[8][d] . X^T[d][8].  The k range is split over the
+//      8 warps; warp w keeps its slice of X as B fragments in registers for the whole pass.  A thread
+//      (row g = lane >> 2, q = lane & 3) loads ONE 16-byte chunk of weight row g per 32 k-values and feeds
+//      its four bf16 pairs to two MMAs; the token rows are chunked the same way, so the k order inside an
+//      MMA is a permutation applied to both operands, which a dot product does not see.  fp32 token rows
+//      are split into a bf16 head and a bf16 remainder (two MMAs).
+//  (2) after an mbarrier over the warps, every warp sums the 8 partial D tiles, forms
+//      h = silu(g) * u * gate weight for the 4 x 8 (unit, token) pairs (one per lane), and
+//  (3) adds h . down rows into the 16-column output blocks it owns: D[16 cols][8 tokens] += A . B with
+//      A = the 4 down rows read transposed by ldmatrix (k = unit, zero-padded to 16), B = h as bf16 head +
+//      remainder.  The accumulators stay in registers for the pass and leave as fixed-point atomics.
+// Units of a stage sit `unit_stride` = 3*d*2 + 16 bytes apart, so the 4 down rows fall into different banks.
+constexpr int kMmaGroups = 8;   // 32-value k groups per warp (d <= 2048)
+constexpr int kMmaBlocks = 16;  // 16-column output blocks per warp (d <= 2048)
+
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(saddr));
+}
+// (a, b) -> bf16 pair `head` (a in the low half) and the pair of what rounding left over
+__device__ __forceinline__ void split_bf16x2(float a, float b, uint32_t& head, uint32_t& rest) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(a - __low2float(h), b - __high2float(h));
+  head = *reinterpret_cast<const uint32_t*>(&h);
+  rest = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+template <bool XBF>  // token rows are bf16 (else fp32: head + remainder)
+__device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm, const Pass& ps, const unsigned char* ring,
+                                                 const unsigned char* xs, RingPos& rp, int warp, int lane) {
   DeviceState* st = P.st;
-  const int NS = P.n_stages, d = P.d, chunks = d >> 3;
+  const int NS = P.n_stages, d = P.d, chunks = d >> 3, cl = chunks - 1;
   const int n = ps.ns;
-  const bool xbf = P.x_is_bf16 != 0;
+  constexpr bool xbf = XBF;
   const int xrow_bytes = d * (xbf ? 2 : 4);
   const int slot0 = sm.act_off[ps.ai] + ps.s0;
-  // output columns this lane owns in step (2): one 8-column chunk
-  const int cw0 = (warp * chunks) / kWarps, cw1 = ((warp + 1) * chunks) / kWarps;
-  const int mychunk = cw0 + lane;
-  const bool owner = mychunk < cw1;
-  const int cclamp = owner ? mychunk : cw0;
-  float acc[NT][8];
+  const int gid = lane >> 2, q = lane & 3;
+  // (1) k groups of 32 values owned by this warp, and its slice of the token rows as B fragments
+  const int G = (chunks + 3) >> 2;
+  const int g_lo = warp * G / kWarps, g_n = (warp + 1) * G / kWarps - g_lo;
+  uint32_t bh[kMmaGroups][4], bl[XBF ? 1 : kMmaGroups][4];
+  {
+    const unsigned char* xr = xs + (size_t)min(gid, n - 1) * xrow_bytes;  // tokens past n: a copy, never used
 #pragma unroll
-  for (int s = 0; s < NT; ++s)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[s][j] = 0.f;
-  float4 xr[NT == 1 ? kXIters : 1][2];
-  const int cl = chunks - 1;
-  if (NT == 1) {
-#pragma unroll
-    for (int it = 0; it < kXIters; ++it) {
-      load_x_chunk(xs, min(lane + 32 * it, cl), xbf, xr[NT == 1 ? it : 0][0], xr[NT == 1 ? it : 0][1]);
-      if (lane + 32 * it > cl) xr[NT == 1 ? it : 0][0] = xr[NT == 1 ? it : 0][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int gi = 0; gi < kMmaGroups; ++gi) {
+      const int cc = min(4 * (g_lo + gi) + q, cl);
+      if (gi < g_n) {
+        if (xbf) {
+          const uint4 v = reinterpret_cast<const uint4*>(xr)[cc];
+          bh[gi][0] = v.x, bh[gi][1] = v.y, bh[gi][2] = v.z, bh[gi][3] = v.w;
+        } else {
+          const float4 a = reinterpret_cast<const float4*>(xr)[2 * cc], b = reinterpret_cast<const float4*>(xr)[2 * cc + 1];
+          constexpr int li = XBF ? 0 : 1;
+          split_bf16x2(a.x, a.y, bh[gi][0], bl[gi * li][0]);
+          split_bf16x2(a.z, a.w, bh[gi][1], bl[gi * li][1]);
+          split_bf16x2(b.x, b.y, bh[gi][2], bl[gi * li][2]);
+          split_bf16x2(b.z, b.w, bh[gi][3], bl[gi * li][3]);
+        }
+      } else {
+        bh[gi][0] = bh[gi][1] = bh[gi][2] = bh[gi][3] = 0u;
+        if (!xbf) bl[XBF ? 0 : gi][0] = bl[XBF ? 0 : gi][1] = bl[XBF ? 0 : gi][2] = bl[XBF ? 0 : gi][3] = 0u;
+      }
     }
   }
-  // gate weight of each token of the pass (1 when the unweighted per-slot output is asked for)
-  const float myw = (lane < n) ? sm.slot_w[slot0 + lane] : 0.f;
+  // (3) output blocks of 16 columns owned by this warp
+  const int NB = (d + 15) >> 4;
+  const int b_lo = warp * NB / kWarps, b_n = (warp + 1) * NB / kWarps - b_lo;
+  float acc[kMmaBlocks][4];
+#pragma unroll
+  for (int b = 0; b < kMmaBlocks; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
+  const float myw = gid < n ? sm.slot_w[slot0 + gid] : 0.f;  // gate weight of token gid
+  const uint32_t zero_addr = (uint32_t)__cvta_generic_to_shared(sm.zero16);
+  // ldmatrix: lane i gives the address of row (i & 7) = unit of matrix (i >> 3): columns 8 * (i >> 3) of a block pair
+  const int lm_unit = lane & 7, lm_col = 8 * (lane >> 3);
 
   for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
     const int nrows = min(kRows, ps.rb - row0);
     if (!mbar_wait(&sm.full[rp.slot], rp.par)) {
-      if (lane == 0) set_abort(st, sm, 0x310u);
+      if (lane == 0) set_abort(st, sm, 0x315u);
       return false;
     }
-    const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * P.stage_bytes);
-    // ---- (1) this warp's dot product: unit (warp >> 1), gate (even warp) or up (odd warp)
-    const int r = warp >> 1;
-    if (r < nrows) {
-      const uint4* wrow = stage + (size_t)(r * 3 + (warp & 1)) * chunks;
-      if (NT == 1) {
-        float a0 = 0.f, a1 = 0.f;
-        {
-          uint4 wv[4];
+    const unsigned char* stage = ring + (size_t)rp.slot * P.stage_bytes;
+    const int buf = rp.n & 1;
+    // ---- (1) partial logits of weight row gid (unit gid >> 1, gate or up) over this warp's k slice
+    {
+      const uint4* arow = reinterpret_cast<const uint4*>(stage + (size_t)min(gid >> 1, nrows - 1) * P.unit_stride) +
+                          (size_t)(gid & 1) * chunks;
+      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int j = 0; j < 4; ++j) wv[j] = wrow[min(lane + 32 * j, cl)];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) dot8(wv[j], xr[NT == 1 ? j : 0][0], xr[NT == 1 ? j : 0][1], a0, a1);
-        }
-        if (chunks > 128) {
-          uint4 wv[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) wv[j] = wrow[min(lane + 32 * (j + 4), cl)];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) dot8(wv[j], xr[NT == 1 ? j + 4 : 0][0], xr[NT == 1 ? j + 4 : 0][1], a0, a1);
-        }
-        const float t = warp_sum(a0 + a1);
-        if (lane == 0) sm.gu[rp.slot][warp][0] = t;
-      } else {
-        float a0[NT], a1[NT];
-#pragma unroll
-        for (int s = 0; s < NT; ++s) a0[s] = 0.f, a1[s] = 0.f;
-        for (int c = lane; c < chunks; c += 32) {
-          const uint4 wv = wrow[c];
-#pragma unroll
-          for (int s = 0; s < NT; ++s) {
-            float4 a, b;
-            load_x_chunk(xs + (size_t)(s < n ? s : n - 1) * xrow_bytes, c, xbf, a, b);
-            dot8(wv, a, b, a0[s], a1[s]);
+      for (int gi = 0; gi < kMmaGroups; ++gi) {
+        if (gi < g_n) {
+          const int c = 4 * (g_lo + gi) + q;
+          uint4 w = arow[min(c, cl)];
+          if (c > cl) w = make_uint4(0u, 0u, 0u, 0u);
+          mma_16816(c0, w.x, 0u, w.y, 0u, bh[gi][0], bh[gi][1]);
+          mma_16816(c1, w.z, 0u, w.w, 0u, bh[gi][2], bh[gi][3]);
+          if (!xbf) {
+            mma_16816(c0, w.x, 0u, w.y, 0u, bl[XBF ? 0 : gi][0], bl[XBF ? 0 : gi][1]);
+            mma_16816(c1, w.z, 0u, w.w, 0u, bl[XBF ? 0 : gi][2], bl[XBF ? 0 : gi][3]);
           }
         }
-#pragma unroll
-        for (int s = 0; s < NT; ++s) {
-          const float t = warp_sum(a0[s] + a1[s]);
-          if (lane == 0 && s < n) sm.gu[rp.slot][warp][s] = t;
-        }
       }
+      // D[row gid][tokens 2q, 2q+1] -> red[buf][gate|up][warp][unit * 8 + token]
+      float* dst = sm.red[buf][gid & 1][warp] + (gid >> 1) * 8 + 2 * q;
+      *reinterpret_cast<float2*>(dst) = make_float2(c0[0] + c1[0], c0[1] + c1[1]);
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.hbar[rp.slot]);
     if (!mbar_wait_spin(&sm.hbar[rp.slot], rp.par)) {
-      if (lane == 0) set_abort(st, sm, 0x311u);
+      if (lane == 0) set_abort(st, sm, 0x316u);
       return false;
     }
-    // ---- (2) h_c for (unit, token) pairs, one per lane, then the rank-1 updates of the owned columns
-    uint4 dw[kRows];
-#pragma unroll
-    for (int rr = 0; rr < kRows; ++rr) dw[rr] = stage[(size_t)(min(rr, nrows - 1) * 3 + 2) * chunks + cclamp];
-    float hv = 0.f;
+    // ---- (2) lane (token gid, unit q): h
+    float h;
     {
-      const int rr = lane / n, s = lane - rr * n;
-      const float wsel = __shfl_sync(0xffffffffu, myw, s);
-      if (rr < nrows) {
-        const float g = sm.gu[rp.slot][2 * rr][s], u = sm.gu[rp.slot][2 * rr + 1][s];
-        hv = g / (1.0f + expf(-g)) * u * wsel;
+      float g = 0.f, u = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        g += sm.red[buf][0][w][q * 8 + gid];
+        u += sm.red[buf][1][w][q * 8 + gid];
       }
+      h = (q < nrows && gid < n) ? g / (1.0f + expf(-g)) * u * myw : 0.f;
     }
+    // B fragment: k = units 2q, 2q+1 (units 4.. are padding), n = token gid
+    uint32_t hb, hr;
+    {
+      const float ha = __shfl_sync(0xffffffffu, h, (lane & ~3) | ((2 * q) & 3));
+      const float hc = __shfl_sync(0xffffffffu, h, (lane & ~3) | ((2 * q + 1) & 3));
+      split_bf16x2(q < 2 ? ha : 0.f, q < 2 ? hc : 0.f, hb, hr);
+    }
+    // ---- (3) this warp's output blocks, two per ldmatrix
+    const uint32_t down0 = (uint32_t)__cvta_generic_to_shared(stage) + (uint32_t)(2 * d * 2);  // down row of unit 0
 #pragma unroll
-    for (int rr = 0; rr < kRows; ++rr) {
-      float w[8];
-      unpack8(dw[rr], w);
-#pragma unroll
-      for (int s = 0; s < NT; ++s) {
-        const float h = __shfl_sync(0xffffffffu, hv, min(rr * n + (s < n ? s : 0), 31));
-        if (s < n && rr < nrows) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) acc[s][j] = fmaf(h, w[j], acc[s][j]);
+    for (int bp = 0; bp < kMmaBlocks; bp += 2) {
+      if (bp < b_n) {
+        const int col = 16 * (b_lo + bp) + lm_col;  // first of the 8 columns this lane's row address covers
+        const bool valid = lm_unit < nrows && col < d && (bp + (lane >> 4)) < b_n;
+        const uint32_t addr = valid ? down0 + (uint32_t)lm_unit * (uint32_t)P.unit_stride + (uint32_t)col * 2u : zero_addr;
+        uint32_t a[4];
+        ldmatrix_x4_trans(a, addr);
+        mma_16816(acc[bp], a[0], a[1], 0u, 0u, hb, 0u);
+        mma_16816(acc[bp], a[0], a[1], 0u, 0u, hr, 0u);
+        if (bp + 1 < b_n) {
+          mma_16816(acc[bp + 1], a[2], a[3], 0u, 0u, hb, 0u);
+          mma_16816(acc[bp + 1], a[2], a[3], 0u, 0u, hr, 0u);
         }
       }
     }
@@ -401,19 +453,116 @@ __device__ __forceinline__ bool consume_pass(const DenseParams& P, Smem& sm, con
     if (lane == 0) mbar_arrive(&sm.freeb[rp.slot]);
     rp.advance(NS);
   }
-  // ---- the pass's partial outputs -> fixed-point accumulators in global memory
-  if (owner) {
+  // ---- the pass's partial outputs -> fixed-point accumulators: acc[b] = (cols 16b + gid, + 8; tokens 2q, 2q+1)
+  {
+    unsigned long long* const acc0 =
+        reinterpret_cast<unsigned long long*>(P.acc) + (size_t)(blockIdx.x % P.acc_copies) * P.acc_copy_stride;
 #pragma unroll
-    for (int s = 0; s < NT; ++s) {
-      if (s < n) {
-        const int gs = slot0 + s;
-        const int rowi = P.mode == 0 ? sm.slot_tok[gs] : gs;
-        unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) +
-                                  (size_t)(blockIdx.x % P.acc_copies) * P.acc_copy_stride + (size_t)rowi * d + mychunk * 8;
+    for (int tt = 0; tt < 2; ++tt) {
+      const int tk = 2 * q + tt;
+      if (tk < n) {
+        const int gs = slot0 + tk;
+        unsigned long long* dst = acc0 + (size_t)(P.mode == 0 ? sm.slot_tok[gs] : gs) * d;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) atomicAdd(dst + j, (unsigned long long)__float2ll_rn(acc[s][j] * kFixScale));
+        for (int b = 0; b < kMmaBlocks; ++b) {
+          if (b < b_n) {
+            const int col = 16 * (b_lo + b) + gid;
+            if (col < d) atomicAdd(dst + col, (unsigned long long)__float2ll_rn(acc[b][tt] * kFixScale));
+            if (col + 8 < d) atomicAdd(dst + col + 8, (unsigned long long)__float2ll_rn(acc[b][2 + tt] * kFixScale));
+          }
+        }
       }
     }
+  }
+  return true;
+}
+
+// One pass with a single token and d > 1024 (the token row, 8 chunks per lane, does not leave room in the
+// registers for a d-wide partial output per warp): per stage (1) warp w takes one of the 8 dot products
+// (unit w >> 1, gate or up), (2) after an mbarrier each lane owns one 8-column chunk of the output and adds
+// the 4 units' h_c * down_c to it.
+__device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm, const Pass& ps, const unsigned char* ring,
+                                                  const unsigned char* xs, RingPos& rp, int warp, int lane) {
+  DeviceState* st = P.st;
+  const int NS = P.n_stages, d = P.d, chunks = d >> 3, cl = chunks - 1;
+  const bool xbf = P.x_is_bf16 != 0;
+  const int slot0 = sm.act_off[ps.ai] + ps.s0;
+  const int cw0 = (warp * chunks) / kWarps, cw1 = ((warp + 1) * chunks) / kWarps;
+  const int mychunk = cw0 + lane;
+  const bool owner = mychunk < cw1;
+  const int cclamp = owner ? mychunk : cw0;
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  float4 xr[kXIters][2];
+#pragma unroll
+  for (int it = 0; it < kXIters; ++it) {
+    load_x_chunk(xs, min(lane + 32 * it, cl), xbf, xr[it][0], xr[it][1]);
+    if (lane + 32 * it > cl) xr[it][0] = xr[it][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const float wgt = sm.slot_w[slot0];
+
+  for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
+    const int nrows = min(kRows, ps.rb - row0);
+    if (!mbar_wait(&sm.full[rp.slot], rp.par)) {
+      if (lane == 0) set_abort(st, sm, 0x310u);
+      return false;
+    }
+    const unsigned char* stage = ring + (size_t)rp.slot * P.stage_bytes;
+    const int r = warp >> 1;
+    if (r < nrows) {
+      const uint4* wrow = reinterpret_cast<const uint4*>(stage + (size_t)r * P.unit_stride) + (size_t)(warp & 1) * chunks;
+      float a0 = 0.f, a1 = 0.f;
+      {
+        uint4 wv[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) wv[j] = wrow[min(lane + 32 * j, cl)];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dot8(wv[j], xr[j][0], xr[j][1], a0, a1);
+      }
+      if (chunks > 128) {
+        uint4 wv[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) wv[j] = wrow[min(lane + 32 * (j + 4), cl)];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dot8(wv[j], xr[j + 4][0], xr[j + 4][1], a0, a1);
+      }
+      const float t = warp_sum(a0 + a1);
+      if (lane == 0) sm.gu[rp.slot][warp] = t;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.hbar[rp.slot]);
+    if (!mbar_wait_spin(&sm.hbar[rp.slot], rp.par)) {
+      if (lane == 0) set_abort(st, sm, 0x311u);
+      return false;
+    }
+    uint4 dw[kRows];
+#pragma unroll
+    for (int rr = 0; rr < kRows; ++rr)
+      dw[rr] = (reinterpret_cast<const uint4*>(stage + (size_t)min(rr, nrows - 1) * P.unit_stride) + 2 * (size_t)chunks)[cclamp];
+    float hv = 0.f;
+    if (lane < nrows) {
+      const float g = sm.gu[rp.slot][2 * lane], u = sm.gu[rp.slot][2 * lane + 1];
+      hv = g / (1.0f + expf(-g)) * u * wgt;
+    }
+#pragma unroll
+    for (int rr = 0; rr < kRows; ++rr) {
+      float w[8];
+      unpack8(dw[rr], w);
+      const float h = __shfl_sync(0xffffffffu, hv, rr);  // 0 for units past nrows
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] = fmaf(h, w[j], acc[j]);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.freeb[rp.slot]);
+    rp.advance(NS);
+  }
+  if (owner) {
+    const int rowi = P.mode == 0 ? sm.slot_tok[slot0] : slot0;
+    unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) +
+                              (size_t)(blockIdx.x % P.acc_copies) * P.acc_copy_stride + (size_t)rowi * d + mychunk * 8;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) atomicAdd(dst + j, (unsigned long long)__float2ll_rn(acc[j] * kFixScale));
   }
   return true;
 }
@@ -447,6 +596,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     fence_proxy_async_smem();
     sm.abort = 0;
     sm.last = 0;
+    sm.zero16[0] = sm.zero16[1] = sm.zero16[2] = sm.zero16[3] = 0u;
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (P.fused_route) {
       // one token: every pass reads token row 0, so the first pass's copy of x can start before the routing
@@ -499,7 +649,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float t = warp_sum(a[j]);
-            if (lane == 0) sm.red[warp][e8 + j] = t;
+            if (lane == 0) sm.rlog[warp][e8 + j] = t;
           }
         }
       } else {
@@ -510,7 +660,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
             a = fmaf(xv, bf16_to_float(__ldg(P.w_router + (size_t)i * E + e)), a);
           }
           a = warp_sum(a);
-          if (lane == 0) sm.red[warp][e] = a;
+          if (lane == 0) sm.rlog[warp][e] = a;
         }
       }
     }
@@ -523,9 +673,9 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     if (warp == 0) {
       float l0 = bias0, l1 = bias1;
       if (lane < P.E)
-        for (int w = 0; w < kWarps; ++w) l0 += sm.red[w][lane];
+        for (int w = 0; w < kWarps; ++w) l0 += sm.rlog[w][lane];
       if (lane + 32 < P.E)
-        for (int w = 0; w < kWarps; ++w) l1 += sm.red[w][lane + 32];
+        for (int w = 0; w < kWarps; ++w) l1 += sm.rlog[w][lane + 32];
       warp_route_finish(l0, l1, P.E, P.k, P.renorm, lane, sm.stage_e, sm.stage_w, nullptr);
       __syncwarp();
       // the k selected experts in ascending order are the active experts, one slot (token 0) each
@@ -681,7 +831,13 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
-        bulk_g2s_hint(ring + (size_t)rp.slot * P.stage_bytes, src, bytes, &sm.full[rp.slot], stream_policy);
+        if (P.use_mma) {  // one copy per hidden unit: the units are padded apart in shared memory
+          for (uint32_t o = 0, u = 0; o < bytes; o += row_bytes, ++u)
+            bulk_g2s_hint(ring + (size_t)rp.slot * P.stage_bytes + (size_t)u * P.unit_stride, src + o, row_bytes,
+                          &sm.full[rp.slot], stream_policy);
+        } else {
+          bulk_g2s_hint(ring + (size_t)rp.slot * P.stage_bytes, src, bytes, &sm.full[rp.slot], stream_policy);
+        }
         copy_mask |= 1u << rp.slot;
         src += bytes;
         rp.advance(NS);
@@ -714,16 +870,13 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         break;
       }
       const unsigned char* xsb = xs + (size_t)b * P.xs_bytes;
-      if (ps.ns == 1 && P.wpart_ok)
+      if (P.use_mma)
+        ok = P.x_is_bf16 ? consume_pass_mma<true>(P, sm, ps, ring, xsb, rp, warp, lane)
+                         : consume_pass_mma<false>(P, sm, ps, ring, xsb, rp, warp, lane);
+      else if (P.wpart_ok)
         ok = consume_pass_t1(P, sm, ps, ring, xsb, wpart, rp, cpar, warp, lane);
-      else if (ps.ns == 1)
-        ok = consume_pass<1>(P, sm, ps, ring, xsb, rp, warp, lane);
-      else if (ps.ns == 2)
-        ok = consume_pass<2>(P, sm, ps, ring, xsb, rp, warp, lane);
-      else if (ps.ns <= 4)
-        ok = consume_pass<4>(P, sm, ps, ring, xsb, rp, warp, lane);
       else
-        ok = consume_pass<8>(P, sm, ps, ring, xsb, rp, warp, lane);
+        ok = consume_pass_cols(P, sm, ps, ring, xsb, rp, warp, lane);
       ++pn;
     }
   }
@@ -805,9 +958,10 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   }
   const int xrow = c.d_model * (P.x_is_bf16 ? 2 : 4);
   P.xs_bytes = (min(T, kMaxN) * xrow + 127) / 128 * 128;
-  P.stage_bytes = kRows * 3 * c.d_model * 2;  // multiple of 16; the ring base is 128-byte aligned
-  P.stage_bytes = (P.stage_bytes + 127) / 128 * 128;
-  P.wpart_ok = c.d_model <= 32 * 8 * kT1Iters ? 1 : 0;
+  P.use_mma = T > 1 ? 1 : 0;
+  P.unit_stride = 3 * c.d_model * 2 + (P.use_mma ? 16 : 0);  // multiple of 16; the ring base is 128-byte aligned
+  P.stage_bytes = (kRows * P.unit_stride + 127) / 128 * 128;
+  P.wpart_ok = (!P.use_mma && c.d_model <= 32 * 8 * kT1Iters) ? 1 : 0;
   const size_t fixed = 2 * (size_t)P.xs_bytes + (P.wpart_ok ? (size_t)kWarps * c.d_model * 4 : 0) + kSmemHeaderBytes + 256;
   const long long avail = (long long)ctx->max_smem_optin - (long long)fixed;
   if (avail < 2ll * P.stage_bytes) return MOE_ERR_UNSUPPORTED;
