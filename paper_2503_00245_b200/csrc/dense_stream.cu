@@ -70,7 +70,7 @@ struct Smem {
   uint64_t xfull[2];           // token rows of a pass landed in xs[0/1]
   uint64_t cbar;               // barrier over the consumer warps
   float gu[kMaxStages][kRows * 2];     // single-token passes at d > 1024: the stage's 8 dot products
-  __align__(16) float red[2][2][kWarps][kRows * 8];  // multi-token passes: [stage parity][gate | up][warp][unit * 8 + token]
+  __align__(16) float red[4][2][kRows * 8][kWarps];  // multi-token passes: [stage index & 3][gate | up][unit * 8 + token][warp]
   __align__(16) uint32_t zero16[4];    // what ldmatrix reads for padding rows
   float rlog[kWarps][MOE_MAX_EXPERTS];
   int act_e[MOE_MAX_EXPERTS];
@@ -300,25 +300,31 @@ __device__ __forceinline__ bool consume_pass_t1(const DenseParams& P, Smem& sm, 
 //      MMA is a permutation applied to both operands, which a dot product does not see.  fp32 token rows
 //      are split into a bf16 head and a bf16 remainder (two MMAs).
 //  (2) after an mbarrier over the warps, every warp sums the 8 partial D tiles, forms
-//      h = silu(g) * u * gate weight for the 4 x 8 (unit, token) pairs (one per lane), and
+//      h = silu(g) * u for the 4 x 8 (unit, token) pairs (one per lane), and
 //  (3) adds h . down rows into the 16-column output blocks it owns: D[16 cols][8 tokens] += A . B with
-//      A = the 4 down rows read transposed by ldmatrix (k = unit, zero-padded to 16), B = h as bf16 head +
-//      remainder.  The accumulators stay in registers for the pass and leave as fixed-point atomics.
+//      A = the 4 down rows read transposed by ldmatrix (k = unit, zero-padded to 8), B = h rounded to bf16
+//      (m16n8k8).  The token's gate weight multiplies the pass's sum at the end.  The accumulators stay in registers for the pass and leave as fixed-point atomics.
 // Units of a stage sit `unit_stride` = 3*d*2 + 16 bytes apart, so the 4 down rows fall into different banks.
-constexpr int kMmaGroups = 8;   // 32-value k groups per warp (d <= 2048)
-constexpr int kMmaBlocks = 16;  // 16-column output blocks per warp (d <= 2048)
+// Template sizes: GROUPS = 32-value k groups per warp, BLOCKS = 16-column output blocks per warp
+// (4 and 8 for d <= 1024, 8 and 16 for d <= 2048).
 
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                           uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_1688(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(b0));
+}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(saddr));
+               : "r"(saddr)
+               : "memory");
 }
 // (a, b) -> bf16 pair `head` (a in the low half) and the pair of what rounding left over
 __device__ __forceinline__ void split_bf16x2(float a, float b, uint32_t& head, uint32_t& rest) {
@@ -328,87 +334,118 @@ __device__ __forceinline__ void split_bf16x2(float a, float b, uint32_t& head, u
   rest = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-template <bool XBF>  // token rows are bf16 (else fp32: head + remainder)
+template <bool XBF, int GROUPS, int BLOCKS>  // XBF: token rows are bf16 (else fp32: head + remainder)
 __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm, const Pass& ps, const unsigned char* ring,
                                                  const unsigned char* xs, RingPos& rp, int warp, int lane) {
   DeviceState* st = P.st;
   const int NS = P.n_stages, d = P.d, chunks = d >> 3, cl = chunks - 1;
   const int n = ps.ns;
-  constexpr bool xbf = XBF;
-  const int xrow_bytes = d * (xbf ? 2 : 4);
+  const int xrow_bytes = d * (XBF ? 2 : 4);
   const int slot0 = sm.act_off[ps.ai] + ps.s0;
   const int gid = lane >> 2, q = lane & 3;
-  // (1) k groups of 32 values owned by this warp, and its slice of the token rows as B fragments
+  // (1) k groups of 32 values owned by this warp: byte offset of this thread's chunk in a row, and its slice of
+  // the token rows as B fragments (zero where the group or the chunk does not exist: the product vanishes
+  // whatever weight bytes are read there)
   const int G = (chunks + 3) >> 2;
   const int g_lo = warp * G / kWarps, g_n = (warp + 1) * G / kWarps - g_lo;
-  uint32_t bh[kMmaGroups][4], bl[XBF ? 1 : kMmaGroups][4];
+  uint32_t coff[GROUPS];
+  uint32_t bh[GROUPS][4], bl[XBF ? 1 : GROUPS][4];
   {
     const unsigned char* xr = xs + (size_t)min(gid, n - 1) * xrow_bytes;  // tokens past n: a copy, never used
 #pragma unroll
-    for (int gi = 0; gi < kMmaGroups; ++gi) {
-      const int cc = min(4 * (g_lo + gi) + q, cl);
-      if (gi < g_n) {
-        if (xbf) {
-          const uint4 v = reinterpret_cast<const uint4*>(xr)[cc];
-          bh[gi][0] = v.x, bh[gi][1] = v.y, bh[gi][2] = v.z, bh[gi][3] = v.w;
-        } else {
-          const float4 a = reinterpret_cast<const float4*>(xr)[2 * cc], b = reinterpret_cast<const float4*>(xr)[2 * cc + 1];
-          constexpr int li = XBF ? 0 : 1;
-          split_bf16x2(a.x, a.y, bh[gi][0], bl[gi * li][0]);
-          split_bf16x2(a.z, a.w, bh[gi][1], bl[gi * li][1]);
-          split_bf16x2(b.x, b.y, bh[gi][2], bl[gi * li][2]);
-          split_bf16x2(b.z, b.w, bh[gi][3], bl[gi * li][3]);
-        }
+    for (int gi = 0; gi < GROUPS; ++gi) {
+      const int c = 4 * (g_lo + gi) + q, cc = min(c, cl);
+      const bool live = gi < g_n && c <= cl;
+      coff[gi] = (uint32_t)cc * 16u;
+      if (XBF) {
+        const uint4 v = reinterpret_cast<const uint4*>(xr)[cc];
+        bh[gi][0] = live ? v.x : 0u, bh[gi][1] = live ? v.y : 0u, bh[gi][2] = live ? v.z : 0u, bh[gi][3] = live ? v.w : 0u;
       } else {
-        bh[gi][0] = bh[gi][1] = bh[gi][2] = bh[gi][3] = 0u;
-        if (!xbf) bl[XBF ? 0 : gi][0] = bl[XBF ? 0 : gi][1] = bl[XBF ? 0 : gi][2] = bl[XBF ? 0 : gi][3] = 0u;
+        float4 a = reinterpret_cast<const float4*>(xr)[2 * cc], b = reinterpret_cast<const float4*>(xr)[2 * cc + 1];
+        if (!live) a = b = make_float4(0.f, 0.f, 0.f, 0.f);
+        constexpr int li = XBF ? 0 : 1;
+        split_bf16x2(a.x, a.y, bh[gi][0], bl[gi * li][0]);
+        split_bf16x2(a.z, a.w, bh[gi][1], bl[gi * li][1]);
+        split_bf16x2(b.x, b.y, bh[gi][2], bl[gi * li][2]);
+        split_bf16x2(b.z, b.w, bh[gi][3], bl[gi * li][3]);
       }
     }
   }
-  // (3) output blocks of 16 columns owned by this warp
+  const uint32_t row_full = (uint32_t)(gid >> 1) * (uint32_t)P.unit_stride + (uint32_t)(gid & 1) * (uint32_t)(2 * d);
+  // (3) output blocks of 16 columns owned by this warp.  ldmatrix: lane i gives the address of row (i & 7) =
+  // hidden unit, for columns 8 * (i >> 3) of a pair of blocks; rows and columns that do not exist read zeros.
   const int NB = (d + 15) >> 4;
   const int b_lo = warp * NB / kWarps, b_n = (warp + 1) * NB / kWarps - b_lo;
-  float acc[kMmaBlocks][4];
+  float acc[BLOCKS][4];
+  uint32_t lmoff[BLOCKS / 2];
+  unsigned lmok = 0;
+  const int lm_unit = lane & 7;
 #pragma unroll
-  for (int b = 0; b < kMmaBlocks; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
-  const float myw = gid < n ? sm.slot_w[slot0 + gid] : 0.f;  // gate weight of token gid
+  for (int b = 0; b < BLOCKS; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f;
+#pragma unroll
+  for (int bp = 0; bp < BLOCKS; bp += 2) {
+    const int col = 16 * (b_lo + bp) + 8 * (lane >> 3);
+    lmoff[bp / 2] = (uint32_t)lm_unit * (uint32_t)P.unit_stride + (uint32_t)(4 * d) + (uint32_t)col * 2u;
+    if (col < d && (bp + (lane >> 4)) < b_n && lm_unit < kRows) lmok |= 1u << (bp / 2);
+  }
   const uint32_t zero_addr = (uint32_t)__cvta_generic_to_shared(sm.zero16);
-  // ldmatrix: lane i gives the address of row (i & 7) = unit of matrix (i >> 3): columns 8 * (i >> 3) of a block pair
-  const int lm_unit = lane & 7, lm_col = 8 * (lane >> 3);
+  const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(ring);
+  float* const red_st = &sm.red[0][gid & 1][(gid >> 1) * 8 + 2 * q][warp];  // + buf * (elements of one buffer)
+  const float* const red_ld = &sm.red[0][0][q * 8 + gid][0];
+  constexpr int kRedBuf = 2 * 32 * kWarps;
 
-  for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
-    const int nrows = min(kRows, ps.rb - row0);
-    if (!mbar_wait(&sm.full[rp.slot], rp.par)) {
+  // gate/up partial logits of one stage -> red[stage index & 3]
+  auto phase1 = [&](const RingPos& r1, int nrows) {
+    const unsigned char* stage = ring + (size_t)r1.slot * P.stage_bytes;
+    const uint32_t rowoff = nrows == kRows ? row_full
+                                           : (uint32_t)min(gid >> 1, nrows - 1) * (uint32_t)P.unit_stride +
+                                                 (uint32_t)(gid & 1) * (uint32_t)(2 * d);
+    const unsigned char* arow = stage + rowoff;
+    uint4 w[GROUPS];
+#pragma unroll
+    for (int gi = 0; gi < GROUPS; ++gi) w[gi] = *reinterpret_cast<const uint4*>(arow + coff[gi]);
+    float c[4][4];  // four independent accumulation chains
+#pragma unroll
+    for (int j = 0; j < 4; ++j) c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
+#pragma unroll
+    for (int gi = 0; gi < GROUPS; ++gi) {
+      mma_16816(c[(2 * gi) & 3], w[gi].x, 0u, w[gi].y, 0u, bh[gi][0], bh[gi][1]);
+      mma_16816(c[(2 * gi + 1) & 3], w[gi].z, 0u, w[gi].w, 0u, bh[gi][2], bh[gi][3]);
+      if (!XBF) {
+        mma_16816(c[(2 * gi + 2) & 3], w[gi].x, 0u, w[gi].y, 0u, bl[XBF ? 0 : gi][0], bl[XBF ? 0 : gi][1]);
+        mma_16816(c[(2 * gi + 3) & 3], w[gi].z, 0u, w[gi].w, 0u, bl[XBF ? 0 : gi][2], bl[XBF ? 0 : gi][3]);
+      }
+    }
+    // D[row gid][tokens 2q, 2q+1] -> red[buf][gate | up][unit * 8 + token][warp]
+    float* dst = red_st + (r1.n & 3) * kRedBuf;
+    dst[0] = (c[0][0] + c[1][0]) + (c[2][0] + c[3][0]);
+    dst[kWarps] = (c[0][1] + c[1][1]) + (c[2][1] + c[3][1]);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.hbar[r1.slot]);
+  };
+
+  // The logits of stage i + 1 are issued before the barrier of stage i is waited for, so the barrier's round
+  // trip and the other warps' skew hide behind tensor-core work.  A warp can be at most two stages behind
+  // another one that is writing `red`, hence its four buffers.
+  RingPos r1 = rp;  // the stage whose logits are computed next
+  if (ps.ra < ps.rb) {
+    if (!mbar_wait(&sm.full[r1.slot], r1.par)) {
       if (lane == 0) set_abort(st, sm, 0x315u);
       return false;
     }
-    const unsigned char* stage = ring + (size_t)rp.slot * P.stage_bytes;
-    const int buf = rp.n & 1;
-    // ---- (1) partial logits of weight row gid (unit gid >> 1, gate or up) over this warp's k slice
-    {
-      const uint4* arow = reinterpret_cast<const uint4*>(stage + (size_t)min(gid >> 1, nrows - 1) * P.unit_stride) +
-                          (size_t)(gid & 1) * chunks;
-      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int gi = 0; gi < kMmaGroups; ++gi) {
-        if (gi < g_n) {
-          const int c = 4 * (g_lo + gi) + q;
-          uint4 w = arow[min(c, cl)];
-          if (c > cl) w = make_uint4(0u, 0u, 0u, 0u);
-          mma_16816(c0, w.x, 0u, w.y, 0u, bh[gi][0], bh[gi][1]);
-          mma_16816(c1, w.z, 0u, w.w, 0u, bh[gi][2], bh[gi][3]);
-          if (!xbf) {
-            mma_16816(c0, w.x, 0u, w.y, 0u, bl[XBF ? 0 : gi][0], bl[XBF ? 0 : gi][1]);
-            mma_16816(c1, w.z, 0u, w.w, 0u, bl[XBF ? 0 : gi][2], bl[XBF ? 0 : gi][3]);
-          }
-        }
+    phase1(r1, min(kRows, ps.rb - ps.ra));
+    r1.advance(NS);
+  }
+  for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
+    const int nrows = min(kRows, ps.rb - row0);
+    if (row0 + kRows < ps.rb) {
+      if (!mbar_wait(&sm.full[r1.slot], r1.par)) {
+        if (lane == 0) set_abort(st, sm, 0x315u);
+        return false;
       }
-      // D[row gid][tokens 2q, 2q+1] -> red[buf][gate|up][warp][unit * 8 + token]
-      float* dst = sm.red[buf][gid & 1][warp] + (gid >> 1) * 8 + 2 * q;
-      *reinterpret_cast<float2*>(dst) = make_float2(c0[0] + c1[0], c0[1] + c1[1]);
+      phase1(r1, min(kRows, ps.rb - row0 - kRows));
+      r1.advance(NS);
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.hbar[rp.slot]);
     if (!mbar_wait_spin(&sm.hbar[rp.slot], rp.par)) {
       if (lane == 0) set_abort(st, sm, 0x316u);
       return false;
@@ -416,37 +453,32 @@ __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm,
     // ---- (2) lane (token gid, unit q): h
     float h;
     {
-      float g = 0.f, u = 0.f;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        g += sm.red[buf][0][w][q * 8 + gid];
-        u += sm.red[buf][1][w][q * 8 + gid];
-      }
-      h = (q < nrows && gid < n) ? g / (1.0f + expf(-g)) * u * myw : 0.f;
+      const float4* rg = reinterpret_cast<const float4*>(red_ld + (rp.n & 3) * kRedBuf);
+      const float4* ru = rg + 32 * kWarps / 4;
+      const float4 g0 = rg[0], g1 = rg[1], u0 = ru[0], u1 = ru[1];
+      const float g = ((g0.x + g0.y) + (g0.z + g0.w)) + ((g1.x + g1.y) + (g1.z + g1.w));
+      const float u = ((u0.x + u0.y) + (u0.z + u0.w)) + ((u1.x + u1.y) + (u1.z + u1.w));
+      h = (q < nrows && gid < n) ? g / (1.0f + __expf(-g)) * u : 0.f;  // the gate weight multiplies the pass's sum
     }
-    // B fragment: k = units 2q, 2q+1 (units 4.. are padding), n = token gid
-    uint32_t hb, hr;
+    // B fragment (k = units 2q, 2q+1 of 8, units 4.. are padding; n = token gid): h rounded to bf16, as the
+    // hidden activations of the tensor-core prefill path are
+    uint32_t hb;
     {
       const float ha = __shfl_sync(0xffffffffu, h, (lane & ~3) | ((2 * q) & 3));
       const float hc = __shfl_sync(0xffffffffu, h, (lane & ~3) | ((2 * q + 1) & 3));
-      split_bf16x2(q < 2 ? ha : 0.f, q < 2 ? hc : 0.f, hb, hr);
+      const __nv_bfloat162 hp = __floats2bfloat162_rn(q < 2 ? ha : 0.f, q < 2 ? hc : 0.f);
+      hb = *reinterpret_cast<const uint32_t*>(&hp);
     }
     // ---- (3) this warp's output blocks, two per ldmatrix
-    const uint32_t down0 = (uint32_t)__cvta_generic_to_shared(stage) + (uint32_t)(2 * d * 2);  // down row of unit 0
+    const uint32_t stage_addr = ring_addr + (uint32_t)rp.slot * (uint32_t)P.stage_bytes;
+    const unsigned ok = lm_unit < nrows ? lmok : 0u;
 #pragma unroll
-    for (int bp = 0; bp < kMmaBlocks; bp += 2) {
+    for (int bp = 0; bp < BLOCKS; bp += 2) {
       if (bp < b_n) {
-        const int col = 16 * (b_lo + bp) + lm_col;  // first of the 8 columns this lane's row address covers
-        const bool valid = lm_unit < nrows && col < d && (bp + (lane >> 4)) < b_n;
-        const uint32_t addr = valid ? down0 + (uint32_t)lm_unit * (uint32_t)P.unit_stride + (uint32_t)col * 2u : zero_addr;
         uint32_t a[4];
-        ldmatrix_x4_trans(a, addr);
-        mma_16816(acc[bp], a[0], a[1], 0u, 0u, hb, 0u);
-        mma_16816(acc[bp], a[0], a[1], 0u, 0u, hr, 0u);
-        if (bp + 1 < b_n) {
-          mma_16816(acc[bp + 1], a[2], a[3], 0u, 0u, hb, 0u);
-          mma_16816(acc[bp + 1], a[2], a[3], 0u, 0u, hr, 0u);
-        }
+        ldmatrix_x4_trans(a, ((ok >> (bp / 2)) & 1u) ? stage_addr + lmoff[bp / 2] : zero_addr);
+        mma_1688(acc[bp], a[0], a[1], hb);
+        mma_1688(acc[bp + 1], a[2], a[3], hb);  // zeros if the block does not exist
       }
     }
     __syncwarp();
@@ -462,13 +494,14 @@ __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm,
       const int tk = 2 * q + tt;
       if (tk < n) {
         const int gs = slot0 + tk;
+        const float wf = sm.slot_w[gs] * kFixScale;  // gate weight of the token (1 for unweighted per-slot output)
         unsigned long long* dst = acc0 + (size_t)(P.mode == 0 ? sm.slot_tok[gs] : gs) * d;
 #pragma unroll
-        for (int b = 0; b < kMmaBlocks; ++b) {
+        for (int b = 0; b < BLOCKS; ++b) {
           if (b < b_n) {
             const int col = 16 * (b_lo + b) + gid;
-            if (col < d) atomicAdd(dst + col, (unsigned long long)__float2ll_rn(acc[b][tt] * kFixScale));
-            if (col + 8 < d) atomicAdd(dst + col + 8, (unsigned long long)__float2ll_rn(acc[b][2 + tt] * kFixScale));
+            if (col < d) atomicAdd(dst + col, (unsigned long long)__float2ll_rn(acc[b][tt] * wf));
+            if (col + 8 < d) atomicAdd(dst + col + 8, (unsigned long long)__float2ll_rn(acc[b][2 + tt] * wf));
           }
         }
       }
@@ -567,6 +600,11 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
   return true;
 }
 
+// One instantiation per kind of pass, so that each gets its own register allocation and a short instruction
+// stream: V_T1 and V_COLS single token (d <= 1024 / larger), V_MMA_* several tokens.
+enum Variant { V_T1 = 0, V_COLS, V_MMA_BF16_S, V_MMA_F32_S, V_MMA_BF16_L, V_MMA_F32_L };
+
+template <int V>
 __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DenseParams P) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
@@ -870,13 +908,18 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         break;
       }
       const unsigned char* xsb = xs + (size_t)b * P.xs_bytes;
-      if (P.use_mma)
-        ok = P.x_is_bf16 ? consume_pass_mma<true>(P, sm, ps, ring, xsb, rp, warp, lane)
-                         : consume_pass_mma<false>(P, sm, ps, ring, xsb, rp, warp, lane);
-      else if (P.wpart_ok)
+      if (V == V_T1)
         ok = consume_pass_t1(P, sm, ps, ring, xsb, wpart, rp, cpar, warp, lane);
-      else
+      else if (V == V_COLS)
         ok = consume_pass_cols(P, sm, ps, ring, xsb, rp, warp, lane);
+      else if (V == V_MMA_BF16_S)
+        ok = consume_pass_mma<true, 4, 8>(P, sm, ps, ring, xsb, rp, warp, lane);
+      else if (V == V_MMA_F32_S)
+        ok = consume_pass_mma<false, 4, 8>(P, sm, ps, ring, xsb, rp, warp, lane);
+      else if (V == V_MMA_BF16_L)
+        ok = consume_pass_mma<true, 8, 16>(P, sm, ps, ring, xsb, rp, warp, lane);
+      else
+        ok = consume_pass_mma<false, 8, 16>(P, sm, ps, ring, xsb, rp, warp, lane);
       ++pn;
     }
   }
@@ -931,6 +974,19 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   }
 }
 
+template <int V>
+int launch_variant(const DenseParams& P, int grid, size_t smem, cudaStream_t s) {
+  MOE_CUDA_TRY(cudaFuncSetAttribute(dense_stream_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3(grid), lc.blockDim = dim3(kThreads), lc.dynamicSmemBytes = smem, lc.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr, lc.numAttrs = 1;
+  MOE_CUDA_TRY(cudaLaunchKernelEx(&lc, dense_stream_kernel<V>, P));
+  return MOE_OK;
+}
+
 }  // namespace
 
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
@@ -968,14 +1024,19 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   P.n_stages = (int)min((long long)kMaxStages, avail / P.stage_bytes);
   const size_t smem = (size_t)P.n_stages * P.stage_bytes + fixed;
   const int G = ctx->sm_count;
-  MOE_CUDA_TRY(cudaFuncSetAttribute(dense_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3(G), lc.blockDim = dim3(kThreads), lc.dynamicSmemBytes = smem, lc.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  lc.attrs = attr, lc.numAttrs = 1;
-  MOE_CUDA_TRY(cudaLaunchKernelEx(&lc, dense_stream_kernel, P));
+  const int v = !P.use_mma ? (P.wpart_ok ? V_T1 : V_COLS)
+                           : (c.d_model <= 1024 ? (P.x_is_bf16 ? V_MMA_BF16_S : V_MMA_F32_S)
+                                                : (P.x_is_bf16 ? V_MMA_BF16_L : V_MMA_F32_L));
+  int rc;
+  switch (v) {
+    case V_T1: rc = launch_variant<V_T1>(P, G, smem, s); break;
+    case V_COLS: rc = launch_variant<V_COLS>(P, G, smem, s); break;
+    case V_MMA_BF16_S: rc = launch_variant<V_MMA_BF16_S>(P, G, smem, s); break;
+    case V_MMA_F32_S: rc = launch_variant<V_MMA_F32_S>(P, G, smem, s); break;
+    case V_MMA_BF16_L: rc = launch_variant<V_MMA_BF16_L>(P, G, smem, s); break;
+    default: rc = launch_variant<V_MMA_F32_L>(P, G, smem, s); break;
+  }
+  if (rc != MOE_OK) return rc;
   ctx->launches++;
   return MOE_OK;
 }
