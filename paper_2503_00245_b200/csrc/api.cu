@@ -252,7 +252,7 @@ int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights*
   char* wsb = (char*)ws;
   int32_t* idx = topk_idx ? topk_idx : (int32_t*)(wsb + L.topk_idx);
   float* wt = topk_w ? topk_w : (float*)(wsb + L.topk_w);
-  if (path == MOE_PATH_STREAM && ctx->cfg.wd_rank == 0 && T == 1)  // the router runs inside the expert kernel
+  if (path == MOE_PATH_STREAM && ctx->cfg.wd_rank == 0 && dense_stream_fuses_route(ctx->cfg, T))  // router inside the expert kernel
     return launch_dense_stream(ctx, 0, x, T, w, idx, wt, nullptr, nullptr, y, nullptr, s);
   rc = launch_route(ctx, x, T, w, idx, wt, nullptr, s);
   if (rc != MOE_OK) return rc;

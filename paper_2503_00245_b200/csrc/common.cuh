@@ -32,7 +32,8 @@ struct DeviceState {
   unsigned int bar_gen;  // generation, bumped by the last arriver (own line: it takes the polling)
   unsigned int pad2[31];
   unsigned int done_count;  // CTAs that have added their partial outputs (dense streaming path)
-  unsigned int pad3[31];
+  unsigned int fin_count;   // finalizer CTAs that have finished their slice (directly after done_count)
+  unsigned int pad3[30];
 };
 
 }  // namespace cosmoe
@@ -79,6 +80,7 @@ int launch_stream_ffn(moe_ctx* ctx, int mode, const void* x, int T, const moe_we
                       char* ws, const WsLayout& L, cudaStream_t s);
 // Dense experts, streaming path, one kernel (router fused when T == 1 and mode == 0; mode 2 = mode 0 with the
 // routing always taken from topk_idx / topk_w).
+bool dense_stream_fuses_route(const moe_config& c, int T);  // mode 0 computes the routing itself (else: run launch_route first)
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
                         float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
                         cudaStream_t s);

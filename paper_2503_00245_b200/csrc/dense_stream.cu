@@ -37,6 +37,7 @@ constexpr int kMaxN = 8;       // tokens of one expert handled per pass over its
 constexpr int kMaxStages = 8;
 constexpr int kXIters = 8;     // 16-byte chunks of x per lane: d <= 2048
 constexpr int kMaxSlots = MOE_STREAM_MAX_TOKENS * MOE_MAX_TOPK;
+constexpr int kFinalizers = 8;  // CTAs that share the conversion of the sums into the output
 constexpr float kFixScale = 68719476736.0f;      // 2^36
 constexpr double kFixInv = 1.0 / 68719476736.0;
 
@@ -615,6 +616,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   const int NS = P.n_stages;
   DeviceState* const st = P.st;
   const int n_pairs = P.T * P.k;
+  const bool fused1 = P.fused_route && P.T == 1;  // one token: the router is spread over the whole CTA
 
   // ------------------------------------------------------------------ prologue
   // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as this one's CTAs
@@ -636,7 +638,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     sm.last = 0;
     sm.zero16[0] = sm.zero16[1] = sm.zero16[2] = sm.zero16[3] = 0u;
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (P.fused_route) {
+    if (fused1) {
       // one token: every pass reads token row 0, so the first pass's copy of x can start before the routing
       const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
       mbar_arrive_expect_tx(&sm.xfull[0], xrow_bytes);
@@ -646,14 +648,14 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   // the router's weights do not depend on any earlier kernel: the first group of eight experts is fetched
   // before the dependency wait, so its DRAM latency overlaps the predecessor's tail
   uint4 wr0[kXIters];
-  const bool prefetched = P.fused_route && warp < kWarps && (P.E & 7) == 0;
+  const bool prefetched = fused1 && warp < kWarps && (P.E & 7) == 0;
   if (prefetched) {
 #pragma unroll
     for (int j = 0; j < kXIters; ++j)
       wr0[j] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + j * kConsumerThreads, P.d - 1) * P.E));
   }
   if (tid != kConsumerThreads) asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (P.fused_route) {
+  if (fused1) {
     // router logits of the single token: every consumer thread takes rows of W_r (row i = the E weights
     // of input feature i), 8 experts at a time
     if (warp < kWarps) {
@@ -738,6 +740,44 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         sm.n_act = P.k;
       }
     }
+  } else if (P.fused_route) {
+    // several tokens, E a multiple of 8: one warp per token (Eq. 2, Eq. 3); every CTA routes all tokens
+    if (warp < kWarps) {
+      const int d = P.d, E = P.E;
+      for (int t = warp; t < P.T; t += kWarps) {
+        float l0 = 0.f, l1 = 0.f;
+        for (int e8 = 0; e8 < E; e8 += 8) {
+          float a[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) a[j] = 0.f;
+#pragma unroll 4
+          for (int i = lane; i < d; i += 32) {
+            const float xv = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[(size_t)t * d + i])
+                                         : ((const float*)P.x)[(size_t)t * d + i];
+            float w[8];
+            unpack8(__ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)i * E + e8)), w);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a[j] = fmaf(xv, w[j], a[j]);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float v = warp_sum(a[j]);
+            if (lane == e8 + j) l0 = v;
+            if (lane + 32 == e8 + j) l1 = v;
+          }
+        }
+        if (P.b_router) {
+          if (lane < E) l0 += P.b_router[lane];
+          if (lane + 32 < E) l1 += P.b_router[lane + 32];
+        }
+        warp_route_finish(l0, l1, E, P.k, P.renorm, lane, sm.stage_e + t * P.k, sm.stage_w + t * P.k, nullptr);
+        __syncwarp();
+        if (blockIdx.x == 0 && lane < P.k) {
+          if (P.topk_idx) P.topk_idx[t * P.k + lane] = sm.stage_e[t * P.k + lane];
+          if (P.topk_w) P.topk_w[t * P.k + lane] = sm.stage_w[t * P.k + lane];
+        }
+      }
+    }
   } else if (P.mode == 0 && warp == 0) {
     for (int p = lane; p < n_pairs; p += 32) {
       sm.stage_e[p] = P.topk_idx[p];
@@ -745,7 +785,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     }
   }
   __syncthreads();
-  if (tid == 0 && !P.fused_route) {
+  if (tid == 0 && !fused1) {
     // routing products -> active experts and their slots (same numbering as moe_permute)
     const int n = n_pairs;
     int na = 0, bad = 0;
@@ -844,7 +884,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       // the pass's token rows (pass 0 of a single-token launch: already on its way since the prologue)
       const int slot0 = sm.act_off[ps.ai] + ps.s0;
       ++pn_issued;
-      if (!(P.fused_route && pn == 0)) {
+      if (!(fused1 && pn == 0)) {
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(&sm.xfull[b], (uint32_t)ps.ns * xrow_bytes);
         for (int s = 0; s < ps.ns; ++s)
@@ -883,7 +923,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       last_idx[b] = rp.n - 1;
       ++pn;
     }
-    if (P.fused_route && pn_issued == 0) (void)mbar_wait(&sm.xfull[0], 0u);  // the early copy of x must land
+    if (fused1 && pn_issued == 0) (void)mbar_wait(&sm.xfull[0], 0u);  // the early copy of x must land
     if (!ok) {
       // copies already in flight must land before this CTA's shared memory goes away
       for (int back = 1; back <= NS && back <= rp.n; ++back) {
@@ -927,33 +967,50 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   // (after an expired wait the warps may be out of step with this barrier: then it can expire too; the
   // status word is already set and nobody finalises)
   bool fin = consumer_sync(sm, cpar, lane);
+  // The last kFinalizers CTAs to arrive turn the fixed-point sums into the output, one slice each, and leave
+  // zeros behind.  All but the very last of them first wait (bounded) for the arrival counter to fill up: the
+  // CTAs they wait for are running or can start on the SMs the finished ones have left.
+  const unsigned G = gridDim.x, K = G < (unsigned)kFinalizers ? G : (unsigned)kFinalizers;
   if (tid == 0) {
     __threadfence();
     const unsigned old = atom_add_acq_rel(&st->done_count, 1u);
-    sm.last = (old == gridDim.x - 1u) ? 1 : 0;
+    int slice = (int)old - (int)(G - K);
+    if (slice >= 0 && old != G - 1u) {
+      const long long t0 = clock64();
+      while (ld_acquire(&st->done_count) < G) {
+        if (clock64() - t0 > kWaitBudgetCycles || sm.abort || ld_acquire(&st->status) != 0u) {
+          flag_error(st, MOE_ERR_TIMEOUT, 0x340u);  // (keeps an earlier error code if one is set)
+          slice = -1;
+          break;
+        }
+      }
+    }
+    sm.last = slice;
     __threadfence();
   }
   fin = consumer_sync(sm, cpar, lane) && fin;
-  if (fin && sm.last) {
-    // the last CTA to arrive turns the fixed-point sums into the output and leaves zeros behind
+  const int slice = sm.last;
+  if (fin && slice >= 0) {
     const int rows = P.mode == 0 ? P.T : n_pairs;
     const long long total = (long long)rows * P.d;
+    const long long per = (total + K - 1) / K;
+    const long long lo = per * slice, hi = lo + per < total ? lo + per : total;
     const bool good = ld_acquire(&st->status) == 0u;
     // four outputs per thread at a time: all their copies are fetched in one round trip, then summed,
     // converted, stored, and the copies zeroed
-    for (long long i0 = tid; i0 < total; i0 += 4 * kConsumerThreads) {
+    for (long long i0 = lo + tid; i0 < hi; i0 += 4 * kConsumerThreads) {
       long long part[4][8];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const long long i = i0 + (long long)j * kConsumerThreads;
 #pragma unroll
         for (int c = 0; c < 8; ++c)
-          part[j][c] = (i < total && c < P.acc_copies) ? __ldcg(P.acc + (size_t)c * P.acc_copy_stride + i) : 0ll;
+          part[j][c] = (i < hi && c < P.acc_copies) ? __ldcg(P.acc + (size_t)c * P.acc_copy_stride + i) : 0ll;
       }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const long long i = i0 + (long long)j * kConsumerThreads;
-        if (i >= total) continue;
+        if (i >= hi) continue;
         long long v = 0;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -970,7 +1027,15 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           ((float*)P.y)[i] = fv;
       }
     }
-    if (tid == 0) st->done_count = 0u;
+    // the finalizer that finishes last re-arms the counters for the next launch
+    fin = consumer_sync(sm, cpar, lane);
+    if (fin && tid == 0) {
+      __threadfence();
+      if (atom_add_acq_rel(&st->fin_count, 1u) == K - 1u) {
+        st->fin_count = 0u;
+        st->done_count = 0u;
+      }
+    }
   }
 }
 
@@ -989,6 +1054,8 @@ int launch_variant(const DenseParams& P, int grid, size_t smem, cudaStream_t s) 
 
 }  // namespace
 
+bool dense_stream_fuses_route(const moe_config& c, int T) { return T == 1 || (c.n_experts & 7) == 0; }
+
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
                         float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
                         cudaStream_t s) {
@@ -999,7 +1066,7 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   DenseParams P{};
   P.T = T, P.k = c.top_k, P.E = c.n_experts, P.d = c.d_model, P.f = c.d_ff, P.mode = mode;
   P.x_is_bf16 = c.x_dtype == MOE_BF16, P.renorm = c.renorm;
-  P.fused_route = (mode == 0 && T == 1 && !routing_given) ? 1 : 0;
+  P.fused_route = (mode == 0 && !routing_given && dense_stream_fuses_route(c, T)) ? 1 : 0;
   P.x = x, P.w_router = (const uint16_t*)w->w_router, P.b_router = w->b_router;
   P.topk_idx = topk_idx, P.topk_w = topk_w, P.offsets = offsets, P.perm = perm;
   P.expert_slot = w->expert_slot, P.gud = (const uint16_t*)w->gud;
@@ -1010,7 +1077,8 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
     P.acc_copy_stride = rows * c.d_model;
     const long long fit = (long long)ctx->acc_elems / P.acc_copy_stride;
     if (fit < 1) return MOE_ERR_UNSUPPORTED;
-    P.acc_copies = (int)(fit < 8 ? fit : 8);
+    const long long want = rows >= 16 ? 1 : (16 / rows < 8 ? 16 / rows : 8);  // rows x copies of about 16 spread the atomics enough
+    P.acc_copies = (int)(fit < want ? fit : want);
   }
   const int xrow = c.d_model * (P.x_is_bf16 ? 2 : 4);
   P.xs_bytes = (min(T, kMaxN) * xrow + 127) / 128 * 128;
@@ -1121,7 +1189,7 @@ extern "C" int moe_layer_forward_static(const moe_config* cfg, const void* x, in
   if (T > 1 && (!topk_idx || !topk_w)) return MOE_ERR_INVALID_ARG;
   // The array keeps what the last call left.  A call that ran to its end leaves the accumulators and the
   // arrival counter at zero, one that was cut short does not: clear the part this call uses, keep the status.
-  MOE_CUDA_TRY(cudaMemsetAsync(&st->done_count, 0, sizeof(unsigned int), s));
+  MOE_CUDA_TRY(cudaMemsetAsync(&st->done_count, 0, 2 * sizeof(unsigned int), s));  // done_count, fin_count
   MOE_CUDA_TRY(cudaMemsetAsync(acc, 0, kStaticAccBytes, s));
   moe_ctx tmp{};  // a view, not a context: nothing here owns memory
   tmp.cfg = *cfg;
@@ -1133,7 +1201,7 @@ extern "C" int moe_layer_forward_static(const moe_config* cfg, const void* x, in
   tmp.h_state = nullptr;
   tmp.acc = acc;
   tmp.acc_elems = kStaticAccBytes / sizeof(long long);
-  if (T > 1) {
+  if (!dense_stream_fuses_route(tmp.cfg, T)) {
     rc = launch_route(&tmp, x, T, w, topk_idx, topk_w, nullptr, s);
     if (rc != MOE_OK) return rc;
   }
