@@ -93,12 +93,12 @@ struct Pass {
 };
 struct PassIt {
   int ai, ai_hi, grp, ngrp, ra, rb;
-  unsigned long long u0, u1;
+  unsigned u0, u1;
 };
 
 __device__ __forceinline__ void item_bounds(const Smem& sm, int f, PassIt& g) {
-  const unsigned long long lo = (unsigned long long)g.ai * f, hi = lo + f;
-  const unsigned long long a = g.u0 > lo ? g.u0 : lo, b = g.u1 < hi ? g.u1 : hi;
+  const unsigned lo = (unsigned)g.ai * (unsigned)f, hi = lo + (unsigned)f;
+  const unsigned a = g.u0 > lo ? g.u0 : lo, b = g.u1 < hi ? g.u1 : hi;
   g.ra = (int)(a - lo);
   g.rb = b > a ? (int)(b - lo) : g.ra;
   const int ne = sm.act_off[g.ai + 1] - sm.act_off[g.ai];
@@ -106,13 +106,29 @@ __device__ __forceinline__ void item_bounds(const Smem& sm, int f, PassIt& g) {
   g.grp = 0;
 }
 __device__ __forceinline__ void pass_init(const Smem& sm, int f, PassIt& g) {
-  const unsigned long long U = (unsigned long long)sm.n_act * f;
-  g.u0 = blockIdx.x * U / gridDim.x;
-  g.u1 = (blockIdx.x + 1ull) * U / gridDim.x;
+  const unsigned G = gridDim.x, b = blockIdx.x, na = (unsigned)sm.n_act;
   g.ra = g.rb = g.grp = g.ngrp = 0;
+  if (na > 0 && na <= 16u && G >= na) {
+    // few active experts: every CTA works for ONE expert (a second pass costs its set-up and its output atomics
+    // again); the first G % na experts get one CTA more than the others
+    const unsigned base = G / na, extra = G % na;
+    unsigned ai, j, c;
+    if (b < extra * (base + 1u)) {
+      ai = b / (base + 1u), j = b % (base + 1u), c = base + 1u;
+    } else {
+      const unsigned b2 = b - extra * (base + 1u);
+      ai = extra + b2 / base, j = b2 % base, c = base;
+    }
+    g.u0 = ai * (unsigned)f + j * (unsigned)f / c;  // j * f < 2^23
+    g.u1 = ai * (unsigned)f + (j + 1u) * (unsigned)f / c;
+  } else {
+    const unsigned U = na * (unsigned)f;  // <= 2^22, and G * U < 2^32 (checked at launch)
+    g.u0 = b * U / G;
+    g.u1 = (b + 1u) * U / G;
+  }
   if (g.u1 > g.u0) {
-    g.ai = (int)(g.u0 / f);
-    g.ai_hi = (int)((g.u1 - 1) / f);
+    g.ai = (int)((unsigned)g.u0 / (unsigned)f);
+    g.ai_hi = (int)((unsigned)(g.u1 - 1) / (unsigned)f);
     item_bounds(sm, f, g);
   } else {
     g.ai = 0;
@@ -648,7 +664,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   // the router's weights do not depend on any earlier kernel: the first group of eight experts is fetched
   // before the dependency wait, so its DRAM latency overlaps the predecessor's tail
   uint4 wr0[kXIters];
-  const bool prefetched = fused1 && warp < kWarps && (P.E & 7) == 0;
+  const bool prefetched = P.fused_route && warp < kWarps && (P.E & 7) == 0;
   if (prefetched) {
 #pragma unroll
     for (int j = 0; j < kXIters; ++j)
@@ -741,36 +757,66 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       }
     }
   } else if (P.fused_route) {
-    // several tokens, E a multiple of 8: one warp per token (Eq. 2, Eq. 3); every CTA routes all tokens
+    // several tokens, E a multiple of 8 (Eq. 2, Eq. 3); every CTA routes all tokens.  A thread owns the input
+    // features tid, tid + 256, ...: their router rows are fetched once and serve every token; the tokens go
+    // four at a time so that all their loads are in flight together.
+    float* part = &sm.red[0][0][0][0];  // [warp][16 tokens][16 experts]: `red` is not in use before the passes
+    constexpr int XJ = (V == V_MMA_BF16_S || V == V_MMA_F32_S) ? 4 : kXIters;  // features per thread
+    constexpr int TC = 32 / XJ;                                                // tokens per round trip
     if (warp < kWarps) {
       const int d = P.d, E = P.E;
+      for (int e8 = 0; e8 < E; e8 += 8) {
+        uint4 wr[XJ];
+#pragma unroll
+        for (int j = 0; j < XJ; ++j)
+          wr[j] = e8 == 0 ? wr0[j]
+                          : __ldg(reinterpret_cast<const uint4*>(P.w_router +
+                                                                 (size_t)min(tid + j * kConsumerThreads, d - 1) * E + e8));
+        for (int t0 = 0; t0 < P.T; t0 += TC) {
+          float xv[TC][XJ];
+#pragma unroll
+          for (int tt = 0; tt < TC; ++tt) {
+            const size_t rowo = (size_t)min(t0 + tt, P.T - 1) * d;
+#pragma unroll
+            for (int j = 0; j < XJ; ++j) {
+              const int i = tid + j * kConsumerThreads;
+              if (i < d)
+                xv[tt][j] = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[rowo + i]) : ((const float*)P.x)[rowo + i];
+              else
+                xv[tt][j] = 0.f;
+            }
+          }
+#pragma unroll
+          for (int tt = 0; tt < TC; ++tt) {
+            float a[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) a[q] = 0.f;
+#pragma unroll
+            for (int j = 0; j < XJ; ++j) {
+              float w[8];
+              unpack8(wr[j], w);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) a[q] = fmaf(xv[tt][j], w[q], a[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float v = warp_sum(a[q]);
+              if (lane == 0 && t0 + tt < P.T) part[(warp * 16 + t0 + tt) * 16 + e8 + q] = v;
+            }
+          }
+        }
+      }
+    }
+    const float bias = (P.b_router && lane < P.E) ? P.b_router[lane] : 0.f;
+    __syncthreads();
+    if (warp < kWarps) {
       for (int t = warp; t < P.T; t += kWarps) {
         float l0 = 0.f, l1 = 0.f;
-        for (int e8 = 0; e8 < E; e8 += 8) {
-          float a[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) a[j] = 0.f;
-#pragma unroll 4
-          for (int i = lane; i < d; i += 32) {
-            const float xv = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[(size_t)t * d + i])
-                                         : ((const float*)P.x)[(size_t)t * d + i];
-            float w[8];
-            unpack8(__ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)i * E + e8)), w);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) a[j] = fmaf(xv, w[j], a[j]);
-          }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float v = warp_sum(a[j]);
-            if (lane == e8 + j) l0 = v;
-            if (lane + 32 == e8 + j) l1 = v;
-          }
+        if (lane < P.E) {
+          for (int w = 0; w < kWarps; ++w) l0 += part[(w * 16 + t) * 16 + lane];
+          l0 += bias;
         }
-        if (P.b_router) {
-          if (lane < E) l0 += P.b_router[lane];
-          if (lane + 32 < E) l1 += P.b_router[lane + 32];
-        }
-        warp_route_finish(l0, l1, E, P.k, P.renorm, lane, sm.stage_e + t * P.k, sm.stage_w + t * P.k, nullptr);
+        warp_route_finish(l0, l1, P.E, P.k, P.renorm, lane, sm.stage_e + t * P.k, sm.stage_w + t * P.k, nullptr);
         __syncwarp();
         if (blockIdx.x == 0 && lane < P.k) {
           if (P.topk_idx) P.topk_idx[t * P.k + lane] = sm.stage_e[t * P.k + lane];
@@ -785,38 +831,62 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     }
   }
   __syncthreads();
-  if (tid == 0 && !fused1) {
-    // routing products -> active experts and their slots (same numbering as moe_permute)
+  if (warp == 0 && !fused1 && P.mode == 0) {
+    // routing products -> active experts and their slots (same numbering as moe_permute): lane e works for
+    // experts e and e + 32
+    const int n = n_pairs, E = P.E;
+    int c0 = 0, c1 = 0, bad = 0;
+    for (int p = 0; p < n; ++p) {
+      const int e = sm.stage_e[p];
+      bad |= (e < 0 || e >= E);
+      c0 += (e == lane);
+      c1 += (e == lane + 32);
+    }
+    int s0 = c0, s1 = c1;  // inclusive scans over the lanes
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v0 = __shfl_up_sync(0xffffffffu, s0, o), v1 = __shfl_up_sync(0xffffffffu, s1, o);
+      if (lane >= o) s0 += v0, s1 += v1;
+    }
+    const int tot0 = __shfl_sync(0xffffffffu, s0, 31);
+    int off0 = s0 - c0, off1 = tot0 + s1 - c1;
+    const unsigned m0 = __ballot_sync(0xffffffffu, c0 > 0), m1 = __ballot_sync(0xffffffffu, c1 > 0);
+    const unsigned below = (1u << lane) - 1u;
+    const int na = __popc(m0) + __popc(m1);
+    int sl0 = lane, sl1 = lane + 32;
+    if (P.expert_slot) {
+      if (c0 > 0) sl0 = P.expert_slot[lane];
+      if (c1 > 0) sl1 = P.expert_slot[lane + 32];
+    }
+    bad |= (c0 > 0 && sl0 < 0) || (c1 > 0 && sl1 < 0);
+    bad = __any_sync(0xffffffffu, bad);
+    if (c0 > 0) {
+      const int a = __popc(m0 & below);
+      sm.act_e[a] = lane, sm.act_off[a] = off0, sm.act_slot[a] = sl0 < 0 ? 0 : sl0;
+    }
+    if (c1 > 0) {
+      const int a = __popc(m0) + __popc(m1 & below);
+      sm.act_e[a] = lane + 32, sm.act_off[a] = off1, sm.act_slot[a] = sl1 < 0 ? 0 : sl1;
+    }
+    if (!bad && (c0 > 0 || c1 > 0)) {
+      for (int p = 0; p < n; ++p) {
+        const int e = sm.stage_e[p];
+        if (e == lane) sm.slot_tok[off0] = p / P.k, sm.slot_w[off0] = sm.stage_w[p], ++off0;
+        if (e == lane + 32) sm.slot_tok[off1] = p / P.k, sm.slot_w[off1] = sm.stage_w[p], ++off1;
+      }
+    }
+    if (lane == 0) {
+      sm.act_off[bad ? 0 : na] = bad ? 0 : n;
+      sm.n_act = bad ? 0 : na;  // every CTA takes the same decision from the same data: no CTA streams anything
+      if (bad) flag_error(st, MOE_ERR_STATE, 0x300u);
+    }
+  }
+  if (tid == 0 && !fused1 && P.mode != 0) {
+    // the caller's grouping (moe_permute's products) -> active experts and their slots
     const int n = n_pairs;
     int na = 0, bad = 0;
     sm.act_off[0] = 0;
-    if (P.mode == 0) {
-      for (int e = 0; e < P.E; ++e) sm.cursor[e] = 0;
-      for (int p = 0; p < n && !bad; ++p) {
-        const int e = sm.stage_e[p];
-        if (e < 0 || e >= P.E)
-          bad = 1;
-        else
-          sm.cursor[e]++;
-      }
-      int off = 0;
-      for (int e = 0; e < P.E && !bad; ++e) {
-        const int cnt = sm.cursor[e];
-        sm.cursor[e] = off;
-        if (cnt) {
-          sm.act_e[na] = e;
-          sm.act_off[na] = off;
-          ++na;
-          off += cnt;
-        }
-      }
-      sm.act_off[na] = off;
-      for (int p = 0; p < n && !bad; ++p) {
-        const int s = sm.cursor[sm.stage_e[p]]++;
-        sm.slot_tok[s] = p / P.k;
-        sm.slot_w[s] = sm.stage_w[p];
-      }
-    } else {
+    {
       for (int e = 0; e < P.E; ++e) {
         const int lo = P.offsets[e], hi = P.offsets[e + 1];
         if (lo < 0 || hi < lo || hi > n) {
@@ -1054,7 +1124,10 @@ int launch_variant(const DenseParams& P, int grid, size_t smem, cudaStream_t s) 
 
 }  // namespace
 
-bool dense_stream_fuses_route(const moe_config& c, int T) { return T == 1 || (c.n_experts & 7) == 0; }
+static_assert(MOE_STREAM_MAX_TOKENS <= 16, "the fused router's staging area holds 16 tokens");
+bool dense_stream_fuses_route(const moe_config& c, int T) {
+  return T == 1 || ((c.n_experts & 7) == 0 && c.n_experts <= 16);  // several tokens: 8 or 16 experts
+}
 
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
                         float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
