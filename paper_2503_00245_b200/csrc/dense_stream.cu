@@ -368,7 +368,8 @@ __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm,
   uint32_t coff[GROUPS];
   uint32_t bh[GROUPS][4], bl[XBF ? 1 : GROUPS][4];
   {
-    const unsigned char* xr = xs + (size_t)min(gid, n - 1) * xrow_bytes;  // tokens past n: a copy, never used
+    // xs holds every token row of the call; tokens past n: a copy, never used
+    const unsigned char* xr = xs + (size_t)sm.slot_tok[slot0 + min(gid, n - 1)] * xrow_bytes;
 #pragma unroll
     for (int gi = 0; gi < GROUPS; ++gi) {
       const int c = 4 * (g_lo + gi) + q, cc = min(c, cl);
@@ -633,6 +634,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   DeviceState* const st = P.st;
   const int n_pairs = P.T * P.k;
   const bool fused1 = P.fused_route && P.T == 1;  // one token: the router is spread over the whole CTA
+  constexpr bool kAllX = V >= V_MMA_BF16_S;       // several tokens: every token row is staged once
 
   // ------------------------------------------------------------------ prologue
   // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as this one's CTAs
@@ -659,6 +661,11 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
       mbar_arrive_expect_tx(&sm.xfull[0], xrow_bytes);
       bulk_g2s(xs, P.x, xrow_bytes, &sm.xfull[0]);
+    } else if (kAllX) {
+      // several tokens: all token rows stay in shared memory for the whole kernel (router and every pass)
+      const uint32_t bytes = (uint32_t)P.T * (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
+      mbar_arrive_expect_tx(&sm.xfull[0], bytes);
+      bulk_g2s(xs, P.x, bytes, &sm.xfull[0]);
     }
   }
   // the router's weights do not depend on any earlier kernel: the first group of eight experts is fetched
@@ -765,6 +772,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     constexpr int TC = 32 / XJ;                                                // tokens per round trip
     if (warp < kWarps) {
       const int d = P.d, E = P.E;
+      if (!mbar_wait(&sm.xfull[0], 0u) && lane == 0) set_abort(st, sm, 0x317u);
       for (int e8 = 0; e8 < E; e8 += 8) {
         uint4 wr[XJ];
 #pragma unroll
@@ -781,7 +789,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
             for (int j = 0; j < XJ; ++j) {
               const int i = tid + j * kConsumerThreads;
               if (i < d)
-                xv[tt][j] = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[rowo + i]) : ((const float*)P.x)[rowo + i];
+                xv[tt][j] = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)xs)[rowo + i]) : ((const float*)xs)[rowo + i];
               else
                 xv[tt][j] = 0.f;
             }
@@ -942,7 +950,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     unsigned copy_mask = 0;
     while (ok && next_pass(sm, P.f, pit, ps)) {
       const int b = pn & 1;
-      if (last_idx[b] > known_free) {
+      if (!kAllX && last_idx[b] > known_free) {
         const int L = last_idx[b];
         if (!mbar_wait(&sm.freeb[L % NS], (unsigned)(L / NS) & 1u)) {
           set_abort(st, sm, 0x331u);
@@ -954,7 +962,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       // the pass's token rows (pass 0 of a single-token launch: already on its way since the prologue)
       const int slot0 = sm.act_off[ps.ai] + ps.s0;
       ++pn_issued;
-      if (!(fused1 && pn == 0)) {
+      if (!kAllX && !(fused1 && pn == 0)) {
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(&sm.xfull[b], (uint32_t)ps.ns * xrow_bytes);
         for (int s = 0; s < ps.ns; ++s)
@@ -993,14 +1001,17 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       last_idx[b] = rp.n - 1;
       ++pn;
     }
-    if (fused1 && pn_issued == 0) (void)mbar_wait(&sm.xfull[0], 0u);  // the early copy of x must land
+    if ((fused1 || kAllX) && pn_issued == 0) (void)mbar_wait(&sm.xfull[0], 0u);  // the early copy of x must land
     if (!ok) {
       // copies already in flight must land before this CTA's shared memory goes away
       for (int back = 1; back <= NS && back <= rp.n; ++back) {
         const int j = rp.n - back;
         if ((copy_mask >> (j % NS)) & 1u) (void)mbar_wait(&sm.full[j % NS], (unsigned)(j / NS) & 1u);
       }
-      for (int q = max(0, pn_issued - 2); q < pn_issued; ++q) (void)mbar_wait(&sm.xfull[q & 1], (unsigned)(q >> 1) & 1u);
+      if (kAllX)
+        (void)mbar_wait(&sm.xfull[0], 0u);
+      else
+        for (int q = max(0, pn_issued - 2); q < pn_issued; ++q) (void)mbar_wait(&sm.xfull[q & 1], (unsigned)(q >> 1) & 1u);
     }
     return;
   }
@@ -1011,8 +1022,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     bool ok = true;
     int pn = 0;
     while (ok && next_pass(sm, P.f, pit, ps)) {
-      const int b = pn & 1;
-      if (!mbar_wait(&sm.xfull[b], (unsigned)(pn >> 1) & 1u)) {
+      const int b = kAllX ? 0 : (pn & 1);
+      if (!mbar_wait(&sm.xfull[b], kAllX ? 0u : ((unsigned)(pn >> 1) & 1u))) {
         if (lane == 0) set_abort(st, sm, 0x312u);
         ok = false;
         break;
@@ -1154,7 +1165,8 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
     P.acc_copies = (int)(fit < want ? fit : want);
   }
   const int xrow = c.d_model * (P.x_is_bf16 ? 2 : 4);
-  P.xs_bytes = (min(T, kMaxN) * xrow + 127) / 128 * 128;
+  P.xs_bytes = T > 1 ? ((T * xrow + 1) / 2 + 127) / 128 * 128   // several tokens: the two buffers together hold all rows
+                     : (xrow + 127) / 128 * 128;
   P.use_mma = T > 1 ? 1 : 0;
   P.unit_stride = 3 * c.d_model * 2 + (P.use_mma ? 16 : 0);  // multiple of 16; the ring base is 128-byte aligned
   P.stage_bytes = (kRows * P.unit_stride + 127) / 128 * 128;
