@@ -843,13 +843,20 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     // routing products -> active experts and their slots (same numbering as moe_permute): lane e works for
     // experts e and e + 32
     const int n = n_pairs, E = P.E;
-    int c0 = 0, c1 = 0, bad = 0;
-    for (int p = 0; p < n; ++p) {
-      const int e = sm.stage_e[p];
-      bad |= (e < 0 || e >= E);
-      c0 += (e == lane);
-      c1 += (e == lane + 32);
+    const unsigned below = (1u << lane) - 1u;
+    int bad = 0;
+    sm.cursor[lane] = 0, sm.cursor[lane + 32] = 0;
+    __syncwarp();
+    // counts: the pairs 32 at a time, one per lane; the first lane of each group of equal experts adds the group
+    for (int p0 = 0; p0 < n; p0 += 32) {
+      const int p = p0 + lane;
+      int e = p < n ? sm.stage_e[p] : -1;
+      if (p < n && (e < 0 || e >= E)) bad = 1, e = -1;
+      const unsigned peers = __match_any_sync(0xffffffffu, e);
+      if (e >= 0 && (peers & below) == 0u) sm.cursor[e] += __popc(peers);
+      __syncwarp();
     }
+    const int c0 = sm.cursor[lane], c1 = sm.cursor[lane + 32];
     int s0 = c0, s1 = c1;  // inclusive scans over the lanes
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -857,9 +864,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       if (lane >= o) s0 += v0, s1 += v1;
     }
     const int tot0 = __shfl_sync(0xffffffffu, s0, 31);
-    int off0 = s0 - c0, off1 = tot0 + s1 - c1;
+    const int off0 = s0 - c0, off1 = tot0 + s1 - c1;
     const unsigned m0 = __ballot_sync(0xffffffffu, c0 > 0), m1 = __ballot_sync(0xffffffffu, c1 > 0);
-    const unsigned below = (1u << lane) - 1u;
     const int na = __popc(m0) + __popc(m1);
     int sl0 = lane, sl1 = lane + 32;
     if (P.expert_slot) {
@@ -876,11 +882,23 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       const int a = __popc(m0) + __popc(m1 & below);
       sm.act_e[a] = lane + 32, sm.act_off[a] = off1, sm.act_slot[a] = sl1 < 0 ? 0 : sl1;
     }
-    if (!bad && (c0 > 0 || c1 > 0)) {
-      for (int p = 0; p < n; ++p) {
-        const int e = sm.stage_e[p];
-        if (e == lane) sm.slot_tok[off0] = p / P.k, sm.slot_w[off0] = sm.stage_w[p], ++off0;
-        if (e == lane + 32) sm.slot_tok[off1] = p / P.k, sm.slot_w[off1] = sm.stage_w[p], ++off1;
+    __syncwarp();
+    sm.cursor[lane] = off0, sm.cursor[lane + 32] = off1;  // next free slot of every expert
+    __syncwarp();
+    if (!bad) {
+      for (int p0 = 0; p0 < n; p0 += 32) {
+        const int p = p0 + lane;
+        const int e = p < n ? sm.stage_e[p] : -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, e);
+        const int base = e >= 0 ? sm.cursor[e] : 0;
+        __syncwarp();
+        if (e >= 0) {
+          const int sl = base + __popc(peers & below);  // pairs of one expert keep their order
+          sm.slot_tok[sl] = p / P.k;
+          sm.slot_w[sl] = sm.stage_w[p];
+          if ((peers & below) == 0u) sm.cursor[e] = base + __popc(peers);
+        }
+        __syncwarp();
       }
     }
     if (lane == 0) {
