@@ -31,8 +31,9 @@ struct DeviceState {
   unsigned int pad1[31];
   unsigned int bar_gen;  // generation, bumped by the last arriver (own line: it takes the polling)
   unsigned int pad2[31];
-  unsigned int done_count;  // CTAs that have added their partial outputs (dense streaming path)
-  unsigned int fin_count;   // finalizer CTAs that have finished their slice (directly after done_count)
+  // dense streaming path: CTAs that have added their partial outputs, over all launches since the state was last
+  // cleared (never reset by the kernels: a launch's arrivals are numbered by the remainder modulo its grid size)
+  unsigned long long done_total;
   unsigned int pad3[30];
 };
 
@@ -206,6 +207,16 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
 }
 __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_acquire64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned long long atom_add_acq_rel64(unsigned long long* p, unsigned long long v) {
+  unsigned long long old;
+  asm volatile("atom.acq_rel.gpu.global.add.u64 %0, [%1], %2;" : "=l"(old) : "l"(p), "l"(v) : "memory");
+  return old;
 }
 __device__ __forceinline__ unsigned atom_add_acq_rel(unsigned* p, unsigned v) {
   unsigned old;

@@ -1072,11 +1072,13 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   const unsigned G = gridDim.x, K = G < (unsigned)kFinalizers ? G : (unsigned)kFinalizers;
   if (tid == 0) {
     __threadfence();
-    const unsigned old = atom_add_acq_rel(&st->done_count, 1u);
+    const unsigned long long old_total = atom_add_acq_rel64(&st->done_total, 1ull);
+    const unsigned old = (unsigned)(old_total % G);  // this CTA's arrival number within the launch
+    const unsigned long long target = old_total - old + G;
     int slice = (int)old - (int)(G - K);
     if (slice >= 0 && old != G - 1u) {
       const long long t0 = clock64();
-      while (ld_acquire(&st->done_count) < G) {
+      while (ld_acquire64(&st->done_total) < target) {
         if (clock64() - t0 > kWaitBudgetCycles || sm.abort || ld_acquire(&st->status) != 0u) {
           flag_error(st, MOE_ERR_TIMEOUT, 0x340u);  // (keeps an earlier error code if one is set)
           slice = -1;
@@ -1124,15 +1126,6 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           ((__nv_bfloat16*)P.y)[i] = __float2bfloat16_rn(fv);
         else
           ((float*)P.y)[i] = fv;
-      }
-    }
-    // the finalizer that finishes last re-arms the counters for the next launch
-    fin = consumer_sync(sm, cpar, lane);
-    if (fin && tid == 0) {
-      __threadfence();
-      if (atom_add_acq_rel(&st->fin_count, 1u) == K - 1u) {
-        st->fin_count = 0u;
-        st->done_count = 0u;
       }
     }
   }
@@ -1292,7 +1285,7 @@ extern "C" int moe_layer_forward_static(const moe_config* cfg, const void* x, in
   if (T > 1 && (!topk_idx || !topk_w)) return MOE_ERR_INVALID_ARG;
   // The array keeps what the last call left.  A call that ran to its end leaves the accumulators and the
   // arrival counter at zero, one that was cut short does not: clear the part this call uses, keep the status.
-  MOE_CUDA_TRY(cudaMemsetAsync(&st->done_count, 0, 2 * sizeof(unsigned int), s));  // done_count, fin_count
+  MOE_CUDA_TRY(cudaMemsetAsync(&st->done_total, 0, sizeof(unsigned long long), s));
   MOE_CUDA_TRY(cudaMemsetAsync(acc, 0, kStaticAccBytes, s));
   moe_ctx tmp{};  // a view, not a context: nothing here owns memory
   tmp.cfg = *cfg;
