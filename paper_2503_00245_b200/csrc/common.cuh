@@ -109,6 +109,24 @@ __device__ __forceinline__ void flag_error(DeviceState* st, unsigned code, unsig
   if (atomicCAS(&st->status, 0u, code) == 0u) st->detail = detail;
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// A kernel launched with launch_pdl may be scheduled while its predecessor in the stream is still running;
+// it must not touch anything the predecessor reads or writes before pdl_wait(), which returns once the
+// predecessor has completed and its writes are visible.  (Without the launch attribute both are no-ops.)
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = grid, lc.blockDim = block, lc.dynamicSmemBytes = smem, lc.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr, lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- mbarrier -----------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

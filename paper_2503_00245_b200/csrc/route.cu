@@ -96,6 +96,67 @@ __global__ void __launch_bounds__(kRouteWarps * 32)
                     probs ? probs + (size_t)t * E : nullptr);
 }
 
+// Many tokens, 8 experts, a router matrix of at most 64 KB: every CTA first copies W_r into shared memory, its
+// 16-byte rows (one input feature each) shifted by 16 bytes per 8 rows so that lanes reading rows 8 apart fall
+// into different banks; then its warps walk the tokens, a lane taking 8 consecutive features per 16-byte load
+// of x.  (The kernel above reads W_r through L1 with 32 cache lines per warp instruction.)
+template <typename XT>
+__global__ void __launch_bounds__(kRouteWarps * 32)
+    route_smem_kernel(const XT* __restrict__ x, const uint16_t* __restrict__ w_router, const float* __restrict__ bias,
+                      int T, int d, int k, int renorm, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
+                      float* __restrict__ probs) {
+  constexpr int E = 8;
+  extern __shared__ __align__(16) unsigned char s_w[];  // row r at byte 16 * (r + r / 8)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  for (int r = threadIdx.x; r < d; r += blockDim.x)
+    *reinterpret_cast<uint4*>(s_w + 16 * (r + (r >> 3))) = __ldg(reinterpret_cast<const uint4*>(w_router) + r);
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // x may come from the kernel before
+  __syncthreads();
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int chunks = d >> 3;
+  const float b0 = (bias && lane < E) ? bias[lane] : 0.f;
+  for (int t = blockIdx.x * kRouteWarps + wib; t < T; t += gridDim.x * kRouteWarps) {
+    const XT* xr = x + (size_t)t * d;
+    float acc[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    for (int cb = lane; cb < chunks; cb += 32 * 8) {
+      float xv[8][8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = cb + 32 * u;
+        if (c < chunks) {
+          load_x8<XT>(xr + c * 8, xv[u]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) xv[u][i] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = min(cb + 32 * u, chunks - 1);  // clamped rows meet zero inputs
+        const unsigned char* rows = s_w + 16 * (9 * c);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float wv[8];
+          unpack8(*reinterpret_cast<const uint4*>(rows + 16 * i), wv);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[j] = fmaf(xv[u][i], wv[j], acc[j]);
+        }
+      }
+    }
+    float l0 = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      const float v = warp_sum(acc[e]);
+      if (lane == e) l0 = v;
+    }
+    l0 += b0;
+    warp_route_finish(l0, 0.f, E, k, renorm, lane, topk_idx + (size_t)t * k, topk_w + (size_t)t * k,
+                      probs ? probs + (size_t)t * E : nullptr);
+  }
+}
+
 // Few tokens (decode): one CTA per token, all 256 threads split the d axis so the weight rows are
 // fetched in a single round trip; warp 0 finishes.
 template <typename XT, int EMAX>
@@ -142,6 +203,22 @@ static int launch_route_t(moe_ctx* ctx, const void* x, int T, const moe_weights*
   const dim3 grid(few ? T : (T + kRouteWarps - 1) / kRouteWarps);
   const XT* xp = (const XT*)x;
   const uint16_t* wr = (const uint16_t*)w->w_router;
+  const size_t staged = 18 * (size_t)c.d_model;  // bytes of the shifted copy of W_r (8 experts)
+  if (!few && c.n_experts == 8 && staged <= 96 * 1024) {
+    MOE_CUDA_TRY(cudaFuncSetAttribute(route_smem_kernel<XT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)staged));
+    const int ctas = (T + kRouteWarps - 1) / kRouteWarps;
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(ctas < 2 * ctx->sm_count ? ctas : 2 * ctx->sm_count), lc.blockDim = block;
+    lc.dynamicSmemBytes = staged, lc.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr, lc.numAttrs = 1;
+    MOE_CUDA_TRY(cudaLaunchKernelEx(&lc, route_smem_kernel<XT>, xp, wr, (const float*)w->b_router, T, c.d_model, c.top_k,
+                                    c.renorm, idx, wt, probs));
+    ctx->launches++;
+    return MOE_OK;
+  }
 #define ROUTE_CASE(EM)                                                                                              \
   do {                                                                                                              \
     if (few)                                                                                                        \
@@ -182,6 +259,8 @@ __global__ void __launch_bounds__(kPermThreads)
   __shared__ int s_base[MOE_MAX_EXPERTS];
   __shared__ int s_wc[kPermThreads / 32][MOE_MAX_EXPERTS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  pdl_wait();
   if (tid < MOE_MAX_EXPERTS) s_base[tid] = 0;
   __syncthreads();
   for (int p = tid; p < n; p += kPermThreads) {
@@ -238,8 +317,8 @@ __global__ void __launch_bounds__(kPermThreads)
 int launch_permute(moe_ctx* ctx, const int32_t* idx, int T, int32_t* offsets, int32_t* perm, int32_t* inv,
                    cudaStream_t s) {
   const moe_config& c = ctx->cfg;
-  permute_kernel<<<1, kPermThreads, 0, s>>>(idx, T * c.top_k, c.n_experts, offsets, perm, inv, ctx->d_state);
-  MOE_CUDA_TRY(cudaGetLastError());
+  MOE_CUDA_TRY(launch_pdl(permute_kernel, dim3(1), dim3(kPermThreads), 0, s, idx, T * c.top_k, c.n_experts, offsets, perm, inv,
+                          ctx->d_state));
   ctx->launches++;
   return MOE_OK;
 }
@@ -251,6 +330,8 @@ __global__ void gather_rows_kernel(const XT* __restrict__ x, const int32_t* __re
                                    int d, uint4* __restrict__ out) {
   const int chunks = d / 8;
   const long long total = (long long)n_slots * chunks;
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const int s = (int)(i / chunks), c = (int)(i % chunks);
@@ -270,11 +351,11 @@ int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_s
   const int block = 256;
   const int grid = (int)((total + block - 1) / block < 148 * 16 ? (total + block - 1) / block : 148 * 16);
   if (c.x_dtype == MOE_F32)
-    gather_rows_kernel<float><<<grid, block, 0, s>>>((const float*)x, perm, n_slots, c.top_k, c.d_model, (uint4*)xperm);
+    MOE_CUDA_TRY(launch_pdl(gather_rows_kernel<float>, dim3(grid), dim3(block), 0, s, (const float*)x, perm, n_slots,
+                            c.top_k, c.d_model, (uint4*)xperm));
   else
-    gather_rows_kernel<__nv_bfloat16>
-        <<<grid, block, 0, s>>>((const __nv_bfloat16*)x, perm, n_slots, c.top_k, c.d_model, (uint4*)xperm);
-  MOE_CUDA_TRY(cudaGetLastError());
+    MOE_CUDA_TRY(launch_pdl(gather_rows_kernel<__nv_bfloat16>, dim3(grid), dim3(block), 0, s, (const __nv_bfloat16*)x, perm,
+                            n_slots, c.top_k, c.d_model, (uint4*)xperm));
   ctx->launches++;
   return MOE_OK;
 }
@@ -286,6 +367,8 @@ __global__ void combine_kernel(const float* __restrict__ out_slots, const float*
                                const int32_t* __restrict__ inv, int T, int k, int d, YT* __restrict__ y) {
   const int quads = d / 4;
   const long long total = (long long)T * quads;
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const int t = (int)(i / quads), q = (int)(i % quads);
@@ -312,10 +395,11 @@ int launch_combine(moe_ctx* ctx, const float* out_slots, const float* wt, const 
   const int block = 256;
   const int grid = (int)((total + block - 1) / block < 148 * 16 ? (total + block - 1) / block : 148 * 16);
   if (c.x_dtype == MOE_F32)
-    combine_kernel<float><<<grid, block, 0, s>>>(out_slots, wt, inv, T, c.top_k, c.d_model, (float*)y);
+    MOE_CUDA_TRY(launch_pdl(combine_kernel<float>, dim3(grid), dim3(block), 0, s, out_slots, wt, inv, T, c.top_k, c.d_model,
+                            (float*)y));
   else
-    combine_kernel<__nv_bfloat16><<<grid, block, 0, s>>>(out_slots, wt, inv, T, c.top_k, c.d_model, (__nv_bfloat16*)y);
-  MOE_CUDA_TRY(cudaGetLastError());
+    MOE_CUDA_TRY(launch_pdl(combine_kernel<__nv_bfloat16>, dim3(grid), dim3(block), 0, s, out_slots, wt, inv, T, c.top_k,
+                            c.d_model, (__nv_bfloat16*)y));
   ctx->launches++;
   return MOE_OK;
 }

@@ -175,14 +175,8 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
   const int num_kb = (P.K + kBK - 1) / kBK;
   const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
 
+  pdl_launch_dependents();
   if (tid == 0) {
-    int run = 0;
-    for (int i = 0; i < P.E; ++i) {
-      sm.tile_prefix[i] = run;
-      const int rows = P.offsets[i + 1] - P.offsets[i];
-      run += rows > 0 ? (rows + P.tile_rows - 1) / P.tile_rows : 0;
-    }
-    sm.tile_prefix[P.E] = run;
     for (int i = 0; i < NS; ++i) {
       mbar_init(&sm.full[i], 1);
       mbar_init(&sm.empty[i], 1);
@@ -198,6 +192,18 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
                  "n"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // everything above touches only this CTA's shared memory and TMEM; the expert offsets and the operands may
+  // come from the kernel before
+  pdl_wait();
+  if (tid == 0) {
+    int run = 0;
+    for (int i = 0; i < P.E; ++i) {
+      sm.tile_prefix[i] = run;
+      const int rows = P.offsets[i + 1] - P.offsets[i];
+      run += rows > 0 ? (rows + P.tile_rows - 1) / P.tile_rows : 0;
+    }
+    sm.tile_prefix[P.E] = run;
   }
   tc_fence_before();
   __syncthreads();
@@ -482,7 +488,7 @@ int launch_gg(moe_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const 
   const long long m_tiles = (n_slots + P.tile_rows - 1) / P.tile_rows + c.n_experts;  // upper bound
   const int grid = (int)std::min<long long>(m_tiles * n_tiles, ctx->sm_count);
   MOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  grouped_gemm_kernel<<<grid, kThreadsGG, smem, s>>>(a0, a1, b, P);
+  MOE_CUDA_TRY(launch_pdl(grouped_gemm_kernel, dim3(grid), dim3(kThreadsGG), smem, s, a0, a1, b, P));
   MOE_CUDA_TRY(cudaGetLastError());
   ctx->launches++;
   return MOE_OK;
