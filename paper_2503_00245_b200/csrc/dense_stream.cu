@@ -770,6 +770,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     float* part = &sm.red[0][0][0][0];  // [warp][16 tokens][16 experts]: `red` is not in use before the passes
     constexpr int XJ = (V == V_MMA_BF16_S || V == V_MMA_F32_S) ? 4 : kXIters;  // features per thread
     constexpr int TC = 32 / XJ;                                                // tokens per round trip
+    __syncthreads();  // the barriers the producer thread initialised are waited on below
     if (warp < kWarps) {
       const int d = P.d, E = P.E;
       if (!mbar_wait(&sm.xfull[0], 0u) && lane == 0) set_abort(st, sm, 0x317u);
