@@ -39,6 +39,12 @@ def shape(d, f, E=8, k=2, r=0, xd="bf16", bias="none", cfg_id=8):
     (shape(256, 512, k=8), 2, STREAM),
     (shape(256, 512, r=64), 16, STREAM),
     (shape(256, 512, r=64, xd="f32"), 7, STREAM),
+    # several tokens through the streaming kernel: every instantiation of the tensor-core pass
+    (W.PHONE, 8, STREAM),                           # d > 1024, bf16 rows
+    (shape(2048, 1024, xd="f32"), 5, STREAM),       # d > 1024, fp32 rows (head + remainder)
+    (shape(1440, 3840), 9, STREAM),                 # d not a multiple of 32 x 8: ragged k groups and column blocks
+    (W.PHONE_OFFLOAD, 16, STREAM),                  # E = 16 routed inside the kernel, experts with more than 8 tokens
+    (shape(256, 512, E=64, k=8), 4, STREAM),        # E = 64: router as its own kernel, many active experts
 ])
 def test_layer_forward_matches_checker(sh, T, path):
     lay, t, host = U.build(sh, T, path=path)
