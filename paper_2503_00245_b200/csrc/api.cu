@@ -39,7 +39,7 @@ WsLayout ws_layout(const moe_config& c, int T) {
   const bool tensor_ok = true;
   L.vec_a = take(stream_ok ? n * 2 * (size_t)c.wd_rank * 4 : 0);
   L.vec_b = take(stream_ok ? n * (size_t)c.d_ff * 4 : 0);
-  L.vec_c = take(stream_ok ? n * (size_t)c.wd_rank * 4 : 0);
+  L.vec_c = take(stream_ok ? n * (size_t)c.wd_rank * 8 * 4 : 0);  // v, in up to 8 segments per value
   L.xperm = take(tensor_ok ? n * (size_t)c.d_model * 2 : 0);
   L.hidden = take(tensor_ok ? n * (size_t)c.d_ff * 2 : 0);
   L.mid_a = take(tensor_ok ? n * 4 * (size_t)c.wd_rank * 2 : 0);  // t_g, t_u as hi + lo bf16 pairs
@@ -254,6 +254,9 @@ int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights*
   float* wt = topk_w ? topk_w : (float*)(wsb + L.topk_w);
   if (path == MOE_PATH_STREAM && ctx->cfg.wd_rank == 0 && dense_stream_fuses_route(ctx->cfg, T))  // router inside the expert kernel
     return launch_dense_stream(ctx, 0, x, T, w, idx, wt, nullptr, nullptr, y, nullptr, s);
+  if (path == MOE_PATH_STREAM && wd_decode_applies(ctx->cfg, T))  // one launch, router included
+    return launch_wd_decode(ctx, x, w, idx, wt, y, (float*)(wsb + L.vec_a), (float*)(wsb + L.vec_b),
+                            (float*)(wsb + L.vec_c), s);
   rc = launch_route(ctx, x, T, w, idx, wt, nullptr, s);
   if (rc != MOE_OK) return rc;
   if (path == MOE_PATH_STREAM) {

@@ -34,7 +34,9 @@ struct DeviceState {
   // dense streaming path: CTAs that have added their partial outputs, over all launches since the state was last
   // cleared (never reset by the kernels: a launch's arrivals are numbered by the remainder modulo its grid size)
   unsigned long long done_total;
-  unsigned int pad3[30];
+  // weight-decomposed decode kernel: arrivals at its meetings between the products, counted the same way
+  unsigned long long phase_total;
+  unsigned int pad3[28];
 };
 
 }  // namespace cosmoe
@@ -76,6 +78,11 @@ int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_s
 
 // Streaming (decode) path.  mode 0: whole layer from topk (writes y); mode 1: FFN per slot from
 // expert_offsets/perm (writes out_slots).
+// Batch-1 decode with weight-decomposed experts in one launch (router included); t, h, vpart: fp32 scratch of
+// k*2r, k*f and k*r*8 values.
+bool wd_decode_applies(const moe_config& c, int T);
+int launch_wd_decode(moe_ctx* ctx, const void* x, const moe_weights* w, int32_t* topk_idx, float* topk_w, void* y,
+                     float* t, float* h, float* vpart, cudaStream_t s);
 int launch_stream_ffn(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, const int32_t* topk_idx,
                       const float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
                       char* ws, const WsLayout& L, cudaStream_t s);
