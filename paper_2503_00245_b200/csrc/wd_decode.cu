@@ -12,8 +12,8 @@
 // product is "one warp per output row, lanes along the row": each output is the work of one warp, written with a
 // plain store -- no atomics, no finalisation, bit-identical from call to call.  The router (Eq. 2, Eq. 3) runs in
 // every CTA's prologue.  Between the products the CTAs meet at an arrival counter in global memory that runs
-// over launches (each meeting is the next gridDim.x arrivals), with a bounded wait: the grid is at most two
-// CTAs per SM of 256 threads, so all of it is resident as soon as a predecessor has drained.
+// over launches (each meeting is the next gridDim.x arrivals), with a bounded wait: the grid is one CTA of 256
+// threads per SM, so all of it is resident as soon as a predecessor has drained.
 // Short rows (v = h dL has only k r of them) are cut into up to 8 segments whose partial sums are added, in
 // order, by the reader.
 #include "common.cuh"
@@ -87,7 +87,7 @@ __device__ __forceinline__ float dot8f(const uint4& w, const float* v) {
   return a;
 }
 
-__global__ void __launch_bounds__(kWdThreads, 2) wd_decode_kernel(const WdParams P) {
+__global__ void __launch_bounds__(kWdThreads) wd_decode_kernel(const WdParams P) {
   extern __shared__ __align__(16) unsigned char wd_smem_raw[];
   WdSmem& sm = *reinterpret_cast<WdSmem*>(wd_smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -316,7 +316,7 @@ int launch_wd_decode(moe_ctx* ctx, const void* x, const moe_weights* w, int32_t*
   int per_sm = 0;
   MOE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, wd_decode_kernel, kWdThreads, smem));
   if (per_sm < 1) return MOE_ERR_UNSUPPORTED;
-  const int grid = (per_sm < 2 ? per_sm : 2) * ctx->sm_count;
+  const int grid = ctx->sm_count;  // one CTA per SM: fewer arrivals at a meeting beat more warps per product
   const int n_warps = grid * kWdWarps;
   int split = n_warps / (c.top_k * c.wd_rank);
   P.split = split < 1 ? 1 : (split > kWdMaxSplit ? kWdMaxSplit : split);
