@@ -44,7 +44,7 @@ WsLayout ws_layout(const moe_config& c, int T) {
   L.hidden = take(tensor_ok ? n * (size_t)c.d_ff * 2 : 0);
   L.mid_a = take(tensor_ok ? n * 4 * (size_t)c.wd_rank * 2 : 0);  // t_g, t_u as hi + lo bf16 pairs
   L.mid_b = take(tensor_ok ? n * 2 * (size_t)c.wd_rank * 2 : 0);  // v as a hi + lo pair
-  L.out_slots = take(n * (size_t)c.d_model * 4);
+  L.out_slots = take(n * (size_t)c.d_model * 4 * (n <= (size_t)kKSplitMaxSlots ? kKSplitMax : 1));  // room for partial-sum planes
   L.total = off + A;
   return L;
 }
@@ -226,7 +226,7 @@ int moe_expert_ffn(moe_ctx* ctx, const void* x, int32_t T, const moe_weights* w,
     return launch_stream_ffn(ctx, 1, x, T, w, nullptr, nullptr, expert_offsets, perm, nullptr, out_slots, (char*)ws, L,
                              s);
   }
-  return launch_tensor_ffn(ctx, x, T, w, expert_offsets, perm, (char*)ws, L, out_slots, s);
+  return launch_tensor_ffn(ctx, x, T, w, expert_offsets, perm, (char*)ws, L, out_slots, nullptr, s);
 }
 
 int moe_combine(moe_ctx* ctx, const float* out_slots, const float* topk_w, const int32_t* inv, int32_t T, void* y,
@@ -234,7 +234,7 @@ int moe_combine(moe_ctx* ctx, const float* out_slots, const float* topk_w, const
   if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
   if (T == 0) return MOE_OK;
   if (!out_slots || !topk_w || !inv || !y || misaligned(out_slots) || misaligned(y)) return MOE_ERR_INVALID_ARG;
-  return launch_combine(ctx, out_slots, topk_w, inv, T, y, (cudaStream_t)stream);
+  return launch_combine(ctx, out_slots, topk_w, inv, T, y, 1, (cudaStream_t)stream);
 }
 
 int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights* w, void* y, int32_t* topk_idx,
@@ -269,9 +269,10 @@ int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights*
   float* out_slots = (float*)(wsb + L.out_slots);
   rc = launch_permute(ctx, idx, T, offsets, perm, inv, s);
   if (rc != MOE_OK) return rc;
-  rc = launch_tensor_ffn(ctx, x, T, w, offsets, perm, wsb, L, out_slots, s);
+  int planes = 1;
+  rc = launch_tensor_ffn(ctx, x, T, w, offsets, perm, wsb, L, out_slots, &planes, s);
   if (rc != MOE_OK) return rc;
-  return launch_combine(ctx, out_slots, wt, inv, T, y, s);
+  return launch_combine(ctx, out_slots, wt, inv, T, y, planes, s);
 }
 
 }  // extern "C"

@@ -72,8 +72,11 @@ int launch_route(moe_ctx* ctx, const void* x, int T, const moe_weights* w, int32
                  cudaStream_t s);
 int launch_permute(moe_ctx* ctx, const int32_t* idx, int T, int32_t* offsets, int32_t* perm, int32_t* inv,
                    cudaStream_t s);
+// out_slots may come as `planes` partial sums, one [T*k][d] plane after the other (summed in order).
+constexpr int kKSplitMax = 4;          // planes the tensor path may ask for ...
+constexpr int kKSplitMaxSlots = 2048;  // ... when there are at most this many (token, choice) slots
 int launch_combine(moe_ctx* ctx, const float* out_slots, const float* wt, const int32_t* inv, int T, void* y,
-                   cudaStream_t s);
+                   int planes, cudaStream_t s);
 int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_slots, void* xperm, cudaStream_t s);
 
 // Streaming (decode) path.  mode 0: whole layer from topk (writes y); mode 1: FFN per slot from
@@ -94,7 +97,8 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
                         cudaStream_t s);
 // Tensor-core (prefill) path: out_slots from x gathered by perm.
 int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, const int32_t* offsets,
-                      const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, cudaStream_t s);
+                      const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, int* out_planes,
+                      cudaStream_t s);
 
 // ------------------------------------------------------------------ device side
 #ifdef __CUDACC__

@@ -364,7 +364,7 @@ int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_s
 // y[t][c] = sum_j w[t][j] * out_slots[inv[t*k+j]][c], j ascending, fp32, one rounding to the output type.
 template <typename YT>
 __global__ void combine_kernel(const float* __restrict__ out_slots, const float* __restrict__ wt,
-                               const int32_t* __restrict__ inv, int T, int k, int d, YT* __restrict__ y) {
+                               const int32_t* __restrict__ inv, int T, int k, int d, int planes, YT* __restrict__ y) {
   const int quads = d / 4;
   const long long total = (long long)T * quads;
   pdl_launch_dependents();
@@ -375,7 +375,12 @@ __global__ void combine_kernel(const float* __restrict__ out_slots, const float*
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int j = 0; j < k; ++j) {
       const float w = wt[(size_t)t * k + j];
-      const float4 o = *reinterpret_cast<const float4*>(out_slots + (size_t)inv[(size_t)t * k + j] * d + q * 4);
+      const float* src = out_slots + (size_t)inv[(size_t)t * k + j] * d + q * 4;
+      float4 o = *reinterpret_cast<const float4*>(src);
+      for (int pl = 1; pl < planes; ++pl) {  // partial sums of a cut contraction, in order
+        const float4 o2 = *reinterpret_cast<const float4*>(src + (size_t)pl * T * k * d);
+        o.x += o2.x, o.y += o2.y, o.z += o2.z, o.w += o2.w;
+      }
       acc.x = fmaf(w, o.x, acc.x), acc.y = fmaf(w, o.y, acc.y), acc.z = fmaf(w, o.z, acc.z), acc.w = fmaf(w, o.w, acc.w);
     }
     if constexpr (sizeof(YT) == 4) {
@@ -389,17 +394,17 @@ __global__ void combine_kernel(const float* __restrict__ out_slots, const float*
 }
 
 int launch_combine(moe_ctx* ctx, const float* out_slots, const float* wt, const int32_t* inv, int T, void* y,
-                   cudaStream_t s) {
+                   int planes, cudaStream_t s) {
   const moe_config& c = ctx->cfg;
   const long long total = (long long)T * (c.d_model / 4);
   const int block = 256;
   const int grid = (int)((total + block - 1) / block < 148 * 16 ? (total + block - 1) / block : 148 * 16);
   if (c.x_dtype == MOE_F32)
     MOE_CUDA_TRY(launch_pdl(combine_kernel<float>, dim3(grid), dim3(block), 0, s, out_slots, wt, inv, T, c.top_k, c.d_model,
-                            (float*)y));
+                            planes, (float*)y));
   else
     MOE_CUDA_TRY(launch_pdl(combine_kernel<__nv_bfloat16>, dim3(grid), dim3(block), 0, s, out_slots, wt, inv, T, c.top_k,
-                            c.d_model, (__nv_bfloat16*)y));
+                            c.d_model, planes, (__nv_bfloat16*)y));
   ctx->launches++;
   return MOE_OK;
 }

@@ -54,6 +54,9 @@ struct GGParams {
   long long ld_out;    // elements
   long long out_off2;  // EPI_BF16_PAIR: column offset of the second half
   long long out_off_lo;  // split: column offset of the remainders
+  int single_a;           // 128-row tiles, one A operand: the stage has no A' part
+  int ksplit;             // the contraction is cut into this many parts, each a work item of its own ...
+  long long plane_elems;  // ... writing its partial sums plane_elems further on in `out` (EPI_F32 only)
   int n_stages;
   DeviceState* st;
 };
@@ -137,13 +140,16 @@ struct SmemGG {
 };
 
 struct Tile {
-  int e, m0, m_end, halves, n0;
+  int e, m0, m_end, halves, n0, ks;
 };
 
 // idx-th tile of this launch: row-tile major, column tile minor (CTAs that run side by side share the A rows
 // and sweep the expert's B columns, which then sit in L2 for the expert's other row tiles).
 __device__ __forceinline__ bool decode_tile(const GGParams& P, const SmemGG& sm, int idx, int n_tiles, Tile& t) {
-  const int mt = idx / n_tiles, nt = idx - mt * n_tiles;
+  const int per_row = n_tiles * P.ksplit;
+  const int mt = idx / per_row, rem = idx - mt * per_row;
+  const int nt = rem / P.ksplit;
+  t.ks = rem - nt * P.ksplit;
   if (mt >= sm.tile_prefix[P.E]) return false;
   int e = 0;
   while (sm.tile_prefix[e + 1] <= mt) ++e;
@@ -167,7 +173,9 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
   // stage layout: [A 16 KB][A' 16 KB][B 32 KB], all 1024-byte aligned (swizzle atoms).  A' is the second
   // 128-row half of the tile, or the second operand (dual_a, 128-row tiles)
   const uint32_t a_bytes = kBM * kBK * 2, b_bytes = 256 * kBK * 2;
-  const uint32_t stage_bytes = 2 * a_bytes + b_bytes;
+  // (tiles of one 128-row half with a single A operand leave A' out: stages of 48 KB, one more of them)
+  const uint32_t n_a = P.single_a ? 1u : 2u;
+  const uint32_t stage_bytes = n_a * a_bytes + b_bytes;
   unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   SmemGG& sm = *reinterpret_cast<SmemGG*>(stages + (size_t)P.n_stages * stage_bytes);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -219,7 +227,8 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       for (int idx = blockIdx.x; ok && decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x) {
         const uint32_t tx = a_bytes * (P.dual_a ? 2 : t.halves) +
                             (P.pair ? 2u * 128u * kBK * 2u : (uint32_t)P.bn * kBK * 2u);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int kb0 = t.ks * num_kb / P.ksplit, kb1 = (t.ks + 1) * num_kb / P.ksplit;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % NS;
           if (it >= NS && !mbar_wait(&sm.empty[s], ((it / NS) - 1) & 1)) {
             flag_error(P.st, MOE_ERR_TIMEOUT, 0x400u);
@@ -229,7 +238,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           }
           unsigned char* st_a0 = stages + (size_t)s * stage_bytes;
           unsigned char* st_a1 = st_a0 + a_bytes;
-          unsigned char* st_b = st_a0 + 2 * a_bytes;
+          unsigned char* st_b = st_a0 + n_a * a_bytes;
           const int k0 = kb * kBK;
           const int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
           mbar_arrive_expect_tx(&sm.full[s], tx);
@@ -270,7 +279,8 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           }
           tc_fence_after();
         }
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int kb0 = t.ks * num_kb / P.ksplit, kb1 = (t.ks + 1) * num_kb / P.ksplit;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % NS;
           if (!mbar_wait(&sm.full[s], (it / NS) & 1)) {
             flag_error(P.st, MOE_ERR_TIMEOUT, 0x401u);
@@ -281,10 +291,10 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           tc_fence_after();
           const uint32_t a0 = smem_u32(stages + (size_t)s * stage_bytes);
           const uint32_t a1 = a0 + a_bytes;
-          const uint32_t b = a0 + 2 * a_bytes;
+          const uint32_t b = a0 + n_a * a_bytes;
 #pragma unroll
           for (int kk = 0; kk < kBK / 16; ++kk) {
-            const bool acc = (kb > 0) || (kk > 0);
+            const bool acc = (kb > kb0) || (kk > 0);
             const uint64_t da0 = smem_desc(a0 + kk * 32, 16, 1024);
             if (P.b_nmajor) {
               const uint64_t db = smem_desc(b + kk * 2048, 64 * kBK * 2, 1024);
@@ -379,7 +389,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
             tc_wait_ld();
             if (!row_ok) continue;
             if (P.epi == EPI_F32) {
-              float* out = (float*)P.out + (size_t)row * P.ld_out + t.n0 + c;
+              float* out = (float*)P.out + (size_t)t.ks * P.plane_elems + (size_t)row * P.ld_out + t.n0 + c;
 #pragma unroll
               for (int v = 0; v < 8; ++v)
                 if (c + 4 * v < ncols)
@@ -476,17 +486,19 @@ int launch_gg(moe_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const 
   const moe_config& c = ctx->cfg;
   P.E = c.n_experts;
   P.st = ctx->d_state;
-  P.n_stages = 3;
-  const size_t stage_bytes = (size_t)kBM * kBK * 2 * 2 + 256 * kBK * 2;
-  const size_t smem = P.n_stages * stage_bytes + sizeof(SmemGG) + 1024 + 128;
-  if ((long long)smem > ctx->max_smem_optin) return MOE_ERR_UNSUPPORTED;
   const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
   // 256-row tiles halve the operand traffic per flop; small problems keep 128-row tiles to fill the SMs
   P.tile_rows = kBM;
   if (!P.dual_a && (long long)((n_slots + kTileRows - 1) / kTileRows) * n_tiles >= 2ll * ctx->sm_count)
     P.tile_rows = kTileRows;
+  P.single_a = (P.tile_rows == kBM && !P.dual_a) ? 1 : 0;
+  P.n_stages = P.single_a ? 4 : 3;
+  const size_t stage_bytes = (size_t)kBM * kBK * 2 * (P.single_a ? 1 : 2) + 256 * kBK * 2;
+  const size_t smem = P.n_stages * stage_bytes + sizeof(SmemGG) + 1024 + 128;
+  if ((long long)smem > ctx->max_smem_optin) return MOE_ERR_UNSUPPORTED;
   const long long m_tiles = (n_slots + P.tile_rows - 1) / P.tile_rows + c.n_experts;  // upper bound
-  const int grid = (int)std::min<long long>(m_tiles * n_tiles, ctx->sm_count);
+  if (P.ksplit < 1) P.ksplit = 1;
+  const int grid = (int)std::min<long long>(m_tiles * n_tiles * P.ksplit, ctx->sm_count);
   MOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   MOE_CUDA_TRY(launch_pdl(grouped_gemm_kernel, dim3(grid), dim3(kThreadsGG), smem, s, a0, a1, b, P));
   MOE_CUDA_TRY(cudaGetLastError());
@@ -503,11 +515,13 @@ int pick_bn(int n_total, int cap) {
 }  // namespace
 
 int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, const int32_t* offsets,
-                      const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, cudaStream_t s) {
+                      const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, int* out_planes,
+                      cudaStream_t s) {
   const moe_config& c = ctx->cfg;
   if (w->expert_slot) return MOE_ERR_UNSUPPORTED;  // the tensor path reads experts in place (slot == expert)
   const int d = c.d_model, f = c.d_ff, r = c.wd_rank, E = c.n_experts;
   const int n_slots = T * c.top_k;
+  if (out_planes) *out_planes = 1;
   void* xperm = ws + L.xperm;
   void* hidden = ws + L.hidden;
   int rc = launch_gather_rows(ctx, x, perm, n_slots, xperm, s);
@@ -527,6 +541,18 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
     if ((rc = make_map_b(&mb, w->gud, d, 3, f, E, 64, kBK)) != MOE_OK) return rc;
     P.K = f, P.n_total = d, P.bn = pick_bn(d, 256), P.pair = 0, P.dual_a = 0, P.b_nmajor = 1, P.b_sub = 2;
     P.epi = EPI_F32, P.out = out_slots, P.ld_out = d, P.out_off2 = 0;
+    if (out_planes && n_slots <= kKSplitMaxSlots) {
+      // short prefill: too few tiles for the SMs, and every tile streams a long run of weights.  The caller
+      // sums planes: cut the contraction so that every SM streams a part, each part into its own plane.
+      const int m_est = std::max((n_slots + kBM - 1) / kBM, std::min(E, n_slots));
+      const long long tiles = (long long)m_est * ((d + P.bn - 1) / P.bn);
+      int ks = (int)(ctx->sm_count / std::max<long long>(tiles, 1));
+      ks = std::min(std::min(ks, kKSplitMax), (f + kBK - 1) / kBK);
+      if (ks > 1) {
+        P.ksplit = ks, P.plane_elems = (long long)n_slots * d;
+        *out_planes = ks;
+      }
+    }
     return launch_gg(ctx, ma, ma, mb, P, n_slots, s);
   }
   // The rank-r intermediates t and v are kept as hi + lo pairs of bf16 (value = hi + lo): the GEMMs that
