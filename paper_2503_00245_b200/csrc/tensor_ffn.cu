@@ -29,7 +29,8 @@ namespace {
 
 constexpr int kBM = 128;  // rows per tile (TMEM lanes)
 constexpr int kBK = 64;   // K elements per stage (128 bytes of bf16 = one swizzle row)
-constexpr int kThreadsGG = 192;
+constexpr int kEpiWarps = 8;  // two per quarter of the TMEM lanes, splitting the columns
+constexpr int kThreadsGG = (2 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;  // two accumulators of 256 columns
 constexpr int kMaxStagesGG = 4;
 constexpr int kTileRows = 2 * kBM;  // rows per tile when the A operand is single (two halves)
@@ -133,7 +134,7 @@ struct SmemGG {
   uint64_t full[kMaxStagesGG];
   uint64_t empty[kMaxStagesGG];
   uint64_t accum_full;   // all MMAs of the current tile have completed
-  uint64_t accum_empty;  // the epilogue has read the accumulators out of TMEM (4 warps arrive)
+  uint64_t accum_empty;  // the epilogue has read the accumulators out of TMEM (all epilogue warps arrive)
   uint32_t tmem_base;
   int abort;
   int tile_prefix[MOE_MAX_EXPERTS + 1];  // row tiles per expert, exclusive scan
@@ -190,7 +191,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       mbar_init(&sm.empty[i], 1);
     }
     mbar_init(&sm.accum_full, 1);
-    mbar_init(&sm.accum_empty, 4);
+    mbar_init(&sm.accum_empty, kEpiWarps);
     sm.abort = 0;
     fence_mbar_init();
     fence_proxy_async_smem();
@@ -318,8 +319,9 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       }
     }
   } else {
-    // ================================================================= epilogue (warps 2..5)
+    // ================================================================= epilogue (warps 2..9)
     const int q = warp & 3;  // TMEM lanes 32q .. 32q+31 are the only ones this warp may read
+    const int cpar = (warp - 2) >> 2;  // which of the two warps of this quarter: it takes every other 32-column chunk
     int tile_i = 0;
     for (int idx = blockIdx.x; decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x, ++tile_i) {
       if (!mbar_wait(&sm.accum_full, tile_i & 1)) {
@@ -334,7 +336,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
         const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(hf * 256);
         if (P.epi == EPI_SWIGLU || P.epi == EPI_BF16_PAIR) {
           __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + t.n0;
-          for (int c = 0; c < P.bn; c += 32) {
+          for (int c = 32 * cpar; c < P.bn; c += 64) {
             uint32_t g[32], u[32];
             tc_ld32(tbase + c, g);
             tc_ld32(tbase + 128 + c, u);
@@ -383,7 +385,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
             }
           }
         } else {
-          for (int c = 0; c < P.bn; c += 32) {
+          for (int c = 32 * cpar; c < P.bn; c += 64) {
             uint32_t a[32];
             tc_ld32(tbase + c, a);
             tc_wait_ld();
