@@ -327,11 +327,12 @@ int launch_permute(moe_ctx* ctx, const int32_t* idx, int T, int32_t* offsets, in
 // xperm[s][:] = bf16(x[perm[s] / k][:])  (operand rows of the tensor-core path, grouped by expert)
 template <typename XT>
 __global__ void gather_rows_kernel(const XT* __restrict__ x, const int32_t* __restrict__ perm, int n_slots, int k,
-                                   int d, uint4* __restrict__ out) {
+                                   int d, uint4* __restrict__ out, DeviceState* st) {
   const int chunks = d / 8;
   const long long total = (long long)n_slots * chunks;
   pdl_launch_dependents();
   pdl_wait();
+  if (blockIdx.x == 0 && threadIdx.x == 0) st->tile_ctr[0] = 0u;  // the first GEMM after this kernel draws its tiles from it
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const int s = (int)(i / chunks), c = (int)(i % chunks);
@@ -352,10 +353,10 @@ int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_s
   const int grid = (int)((total + block - 1) / block < 148 * 16 ? (total + block - 1) / block : 148 * 16);
   if (c.x_dtype == MOE_F32)
     MOE_CUDA_TRY(launch_pdl(gather_rows_kernel<float>, dim3(grid), dim3(block), 0, s, (const float*)x, perm, n_slots,
-                            c.top_k, c.d_model, (uint4*)xperm));
+                            c.top_k, c.d_model, (uint4*)xperm, ctx->d_state));
   else
     MOE_CUDA_TRY(launch_pdl(gather_rows_kernel<__nv_bfloat16>, dim3(grid), dim3(block), 0, s, (const __nv_bfloat16*)x, perm,
-                            n_slots, c.top_k, c.d_model, (uint4*)xperm));
+                            n_slots, c.top_k, c.d_model, (uint4*)xperm, ctx->d_state));
   ctx->launches++;
   return MOE_OK;
 }

@@ -29,6 +29,7 @@ namespace {
 
 constexpr int kBM = 128;  // rows per tile (TMEM lanes)
 constexpr int kBK = 64;   // K elements per stage (128 bytes of bf16 = one swizzle row)
+constexpr int kTileQueue = 8;  // tile indices in flight between the producer and the other roles
 constexpr int kEpiWarps = 8;  // two per quarter of the TMEM lanes, splitting the columns
 constexpr int kThreadsGG = (2 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;  // two accumulators of 256 columns
@@ -55,6 +56,7 @@ struct GGParams {
   long long ld_out;    // elements
   long long out_off2;  // EPI_BF16_PAIR: column offset of the second half
   long long out_off_lo;  // split: column offset of the remainders
+  int ctr_idx;            // which word of DeviceState::tile_ctr hands out this launch's tiles (the other is cleared)
   int single_a;           // 128-row tiles, one A operand: the stage has no A' part
   int ksplit;             // the contraction is cut into this many parts, each a work item of its own ...
   long long plane_elems;  // ... writing its partial sums plane_elems further on in `out` (EPI_F32 only)
@@ -135,6 +137,9 @@ struct SmemGG {
   uint64_t empty[kMaxStagesGG];
   uint64_t accum_full;   // all MMAs of the current tile have completed
   uint64_t accum_empty;  // the epilogue has read the accumulators out of TMEM (all epilogue warps arrive)
+  uint64_t tq_full[kTileQueue];   // the producer has put a tile index into tq[i]
+  uint64_t tq_empty[kTileQueue];  // the MMA thread and every epilogue warp have read it
+  int tq[kTileQueue];
   uint32_t tmem_base;
   int abort;
   int tile_prefix[MOE_MAX_EXPERTS + 1];  // row tiles per expert, exclusive scan
@@ -190,6 +195,10 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       mbar_init(&sm.full[i], 1);
       mbar_init(&sm.empty[i], 1);
     }
+    for (int i = 0; i < kTileQueue; ++i) {
+      mbar_init(&sm.tq_full[i], 1);
+      mbar_init(&sm.tq_empty[i], 1 + kEpiWarps);
+    }
     mbar_init(&sm.accum_full, 1);
     mbar_init(&sm.accum_empty, kEpiWarps);
     sm.abort = 0;
@@ -206,6 +215,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
   // come from the kernel before
   pdl_wait();
   if (tid == 0) {
+    if (blockIdx.x == 0) P.st->tile_ctr[P.ctr_idx ^ 1] = 0u;  // for the next GEMM of the chain (it starts after this one ends)
     int run = 0;
     for (int i = 0; i < P.E; ++i) {
       sm.tile_prefix[i] = run;
@@ -225,7 +235,20 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
     if (lane == 0) {
       int it = 0;  // k-blocks issued so far, over all tiles
       bool ok = true;
-      for (int idx = blockIdx.x; ok && decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x) {
+      // Tiles are drawn from a counter in global memory (the CTAs' tiles differ in cost: one or two halves, operands
+      // found in L2 or not) and passed on to the MMA thread and the epilogue warps through a small queue.
+      for (int ti = 0; ok; ++ti) {
+        const int qs = ti % kTileQueue;
+        if (ti >= kTileQueue && !mbar_wait(&sm.tq_empty[qs], ((ti / kTileQueue) - 1) & 1)) {
+          flag_error(P.st, MOE_ERR_TIMEOUT, 0x404u);
+          sm.abort = 1;
+          ok = false;
+          break;
+        }
+        const int idx = (int)atomicAdd(&P.st->tile_ctr[P.ctr_idx], 1u);
+        sm.tq[qs] = idx;
+        mbar_arrive(&sm.tq_full[qs]);
+        if (!decode_tile(P, sm, idx, n_tiles, t)) break;  // past the last tile: the others stop on it too
         const uint32_t tx = a_bytes * (P.dual_a ? 2 : t.halves) +
                             (P.pair ? 2u * 128u * kBK * 2u : (uint32_t)P.bn * kBK * 2u);
         const int kb0 = t.ks * num_kb / P.ksplit, kb1 = (t.ks + 1) * num_kb / P.ksplit;
@@ -270,7 +293,17 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       const uint32_t idesc_single = instr_desc(P.pair ? 256 : P.bn, P.b_nmajor != 0);
       int it = 0, tile_i = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; ok && decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x, ++tile_i) {
+      for (;; ++tile_i) {
+        const int qs = tile_i % kTileQueue;
+        if (!ok) break;
+        if (!mbar_wait(&sm.tq_full[qs], (tile_i / kTileQueue) & 1)) {
+          flag_error(P.st, MOE_ERR_TIMEOUT, 0x405u);
+          sm.abort = 1;
+          break;
+        }
+        const int idx = sm.tq[qs];
+        mbar_arrive(&sm.tq_empty[qs]);
+        if (!decode_tile(P, sm, idx, n_tiles, t)) break;
         if (tile_i > 0) {  // the previous tile's accumulators must have left TMEM
           if (!mbar_wait(&sm.accum_empty, (tile_i - 1) & 1)) {
             flag_error(P.st, MOE_ERR_TIMEOUT, 0x403u);
@@ -323,7 +356,16 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
     const int q = warp & 3;  // TMEM lanes 32q .. 32q+31 are the only ones this warp may read
     const int cpar = (warp - 2) >> 2;  // which of the two warps of this quarter: it takes every other 32-column chunk
     int tile_i = 0;
-    for (int idx = blockIdx.x; decode_tile(P, sm, idx, n_tiles, t); idx += gridDim.x, ++tile_i) {
+    for (;; ++tile_i) {
+      const int qs = tile_i % kTileQueue;
+      if (!mbar_wait(&sm.tq_full[qs], (tile_i / kTileQueue) & 1)) {
+        if (lane == 0) flag_error(P.st, MOE_ERR_TIMEOUT, 0x406u);
+        break;
+      }
+      const int idx = sm.tq[qs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.tq_empty[qs]);
+      if (!decode_tile(P, sm, idx, n_tiles, t)) break;
       if (!mbar_wait(&sm.accum_full, tile_i & 1)) {
         if (lane == 0) flag_error(P.st, MOE_ERR_TIMEOUT, 0x402u);
         break;
@@ -537,6 +579,7 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
     if ((rc = make_map_b(&mb, w->gud, d, 3, f, E, kBK, 128)) != MOE_OK) return rc;
     P.K = d, P.n_total = f, P.bn = 128, P.pair = 1, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_SWIGLU;
     P.out = hidden, P.ld_out = f, P.out_off2 = 0;
+    P.ctr_idx = 0;
     if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
     // (2) out_slots = hidden Wd   (B = down rows of gud: [k = hidden unit][n = model column], n contiguous)
     if ((rc = make_map_a(&ma, hidden, n_slots, f, f)) != MOE_OK) return rc;
@@ -555,6 +598,7 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
         *out_planes = ks;
       }
     }
+    P.ctr_idx = 1;
     return launch_gg(ctx, ma, ma, mb, P, n_slots, s);
   }
   // The rank-r intermediates t and v are kept as hi + lo pairs of bf16 (value = hi + lo): the GEMMs that
@@ -569,6 +613,7 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
   if ((rc = make_map_b(&mb, w->wd_a, d, 2, r, E, kBK, 128)) != MOE_OK) return rc;
   P.K = d, P.n_total = r, P.bn = 128, P.pair = 1, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_BF16_PAIR;
   P.k_wrap = 0, P.split = split, P.out = mid_a, P.ld_out = 2 * tw, P.out_off2 = tw, P.out_off_lo = r;
+  P.ctr_idx = 0;
   if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (2) hidden = silu(Tg gR) * (Tu uR)
   if ((rc = make_map_a(&ma, mid_a, n_slots, tw, 2 * tw)) != MOE_OK) return rc;
@@ -576,6 +621,7 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
   if ((rc = make_map_b(&mb, w->wd_b, r, 2, f, E, kBK, 128)) != MOE_OK) return rc;
   P.K = tw, P.n_total = f, P.bn = 128, P.pair = 1, P.dual_a = 1, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_SWIGLU;
   P.k_wrap = split ? r : 0, P.split = 0, P.out = hidden, P.ld_out = f, P.out_off2 = 0, P.out_off_lo = 0;
+  P.ctr_idx = 1;
   if ((rc = launch_gg(ctx, ma, ma1, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (3) V = hidden dL
   if ((rc = make_map_a(&ma, hidden, n_slots, f, f)) != MOE_OK) return rc;
@@ -583,6 +629,7 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
   if ((rc = make_map_b(&mb, w->wd_c, f, 1, r, E, kBK, P.bn)) != MOE_OK) return rc;
   P.K = f, P.n_total = r, P.pair = 0, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_BF16;
   P.k_wrap = 0, P.split = split, P.out = mid_b, P.ld_out = tw, P.out_off2 = 0, P.out_off_lo = r;
+  P.ctr_idx = 0;
   if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (4) out_slots = V dR
   if ((rc = make_map_a(&ma, mid_b, n_slots, tw, tw)) != MOE_OK) return rc;
@@ -590,6 +637,7 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
   if ((rc = make_map_b(&mb, w->wd_d, r, 1, d, E, kBK, P.bn)) != MOE_OK) return rc;
   P.K = tw, P.n_total = d, P.pair = 0, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_F32;
   P.k_wrap = split ? r : 0, P.split = 0, P.out = out_slots, P.ld_out = d, P.out_off2 = 0, P.out_off_lo = 0;
+  P.ctr_idx = 1;
   return launch_gg(ctx, ma, ma, mb, P, n_slots, s);
 }
 
