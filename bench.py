@@ -43,6 +43,18 @@ WORKLOADS = {
 }
 DEFAULT = "wearable-decode-T1"
 
+# Shape sweep (--sweep): batch-1 decode over the paper's ablation grid -- active experts k in {1, 2, 4, 8} at E = 8,
+# total experts E in {2, 4, 8, 16} at k = 2 (Fig. 7: time grows with k, not with E) -- and the paper's own layer
+# widths (Table 1).  Reported under "sweep"; not part of --all.
+SWEEP = {}
+for _k in (1, 2, 4, 8):
+    SWEEP[f"sweep-k{_k}-E8"] = (W.WEARABLE.with_(name=f"wearable k={_k} E=8", top_k=_k), 1, "decode")
+for _E in (2, 4, 16):
+    SWEEP[f"sweep-k2-E{_E}"] = (W.WEARABLE.with_(name=f"wearable k=2 E={_E}", n_experts=_E), 1, "decode")
+SWEEP["sweep-d1440-f3840"] = (W.LayerShape("paper phone widths", 8, 1440, 3840), 1, "decode")
+SWEEP["sweep-d432-f1280"] = (W.LayerShape("paper wearable widths", 8, 432, 1280), 1, "decode")
+WORKLOADS.update(SWEEP)
+
 
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -441,6 +453,7 @@ def main():
     ap.add_argument("--slots", type=int, default=4, help="phone-offload-stack: resident experts per layer")
     ap.add_argument("--decode-steps", type=int, default=256, help="phone-offload-stack: tokens")
     ap.add_argument("--all", action="store_true", help="also time the other workloads (reported under 'others')")
+    ap.add_argument("--sweep", action="store_true", help="also time the shape sweep (reported under 'sweep')")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ring", type=int, default=0, help="override the number of distinct layers in the ring")
@@ -489,10 +502,10 @@ def main():
 
     others = []
     if a.all and rank == 0 and world == 1:
-        del res["ring"]
+        res.pop("ring", None)
         torch.cuda.empty_cache()
         for name in WORKLOADS:
-            if name == a.workload:
+            if name == a.workload or name in SWEEP:
                 continue
             try:
                 r = time_workload(name, a.steps, a.warmup, device, rank, 1)
@@ -503,6 +516,22 @@ def main():
             others.append({"workload": name, "metric": m, "value": round(v, 3), "unit": u,
                            "ms_per_step": round(r["ms_per_step"], 5), "launch_mode": r["launch_mode"],
                            "active_experts_per_step": r["active_experts_per_step"], "roofline": roofline(r)})
+            del r
+            torch.cuda.empty_cache()
+
+    sweep = []
+    if a.sweep and rank == 0 and world == 1:
+        res.pop("ring", None)
+        torch.cuda.empty_cache()
+        for name in SWEEP:
+            try:
+                r = time_workload(name, min(a.steps, 1024), a.warmup, device, rank, 1)
+            except Exception as e:  # noqa: BLE001
+                sweep.append({"workload": name, "error": str(e)[:200]})
+                continue
+            rf = roofline(r)
+            sweep.append({"workload": name, "shape": W.describe(r["shape"]), "us_per_token": round(r["ms_per_step"] * 1e3, 3),
+                          "GB_per_s": rf["achieved"], "frac": rf["frac"]})
             del r
             torch.cuda.empty_cache()
 
@@ -526,6 +555,8 @@ def main():
             line["cpu_baseline"] = cpu_baseline(a.workload)
         if others:
             line["others"] = others
+        if sweep:
+            line["sweep"] = sweep
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()

@@ -45,6 +45,13 @@ def shape(d, f, E=8, k=2, r=0, xd="bf16", bias="none", cfg_id=8):
     (shape(1440, 3840), 9, STREAM),                 # d not a multiple of 32 x 8: ragged k groups and column blocks
     (W.PHONE_OFFLOAD, 16, STREAM),                  # E = 16 routed inside the kernel, experts with more than 8 tokens
     (shape(256, 512, E=64, k=8), 4, STREAM),        # E = 64: router as its own kernel, many active experts
+    # the paper's ablation grid (Fig. 7): active experts 1..8 of 8, total experts 2..16 with 2 active
+    (shape(256, 512, E=8, k=4), 1, 0),
+    (shape(256, 512, E=8, k=8), 1, 0),
+    (shape(256, 512, E=2, k=2), 1, 0),
+    (shape(256, 512, E=4, k=2), 3, 0),
+    (shape(256, 512, E=16, k=2), 6, 0),
+    (shape(256, 512, E=2, k=1), 40, 0),             # tensor path with two experts
 ])
 def test_layer_forward_matches_checker(sh, T, path):
     lay, t, host = U.build(sh, T, path=path)
