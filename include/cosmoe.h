@@ -214,6 +214,16 @@ int moe_offload_stats(moe_offload* off, uint64_t* fetches, uint64_t* bytes, uint
 int moe_stack_decode_step(moe_offload* off, moe_ctx* ctx, const moe_weights* routers, float* h,
                           int32_t* topk_trace_host, void* ws, size_t ws_bytes, void* stream);
 
+/* The same step with the expert set of every layer prescribed by the caller
+ * (sel_host [n_layers][k], distinct experts per layer): the layer's gate weights are
+ * the router's probabilities (Eq. 2) of those experts, renormalised over the set.  For
+ * replaying routing traces, e.g. traces with a given expert replacement ratio (Eq. 4-5)
+ * under the rule of Eq. 8.  Because the host knows the sets, it does not wait for the
+ * device between layers: a layer's misses are copied on the offload's copy stream while
+ * earlier layers compute.  Synchronises `stream` once, at the end.                      */
+int moe_stack_decode_step_trace(moe_offload* off, moe_ctx* ctx, const moe_weights* routers, float* h,
+                                const int32_t* sel_host, void* ws, size_t ws_bytes, void* stream);
+
 /* ---- routing-trace metrics (Eq. 4-5, Section 2.3 / 3.3) ---------------------------
  * topk_trace dev [B][T][k] int32.  Writes H (Eq. 4, summed over experts) to
  * h_total_out dev [1] uint64; replacements = H / 2 and H_norm = (H/2) / (B k (T-1)). */

@@ -65,6 +65,8 @@ _SIGS = {
     "moe_offload_resident": (C.c_int, [_P, C.c_int32, C.POINTER(C.c_int32)]),
     "moe_offload_stats": (C.c_int, [_P, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]),
     "moe_stack_decode_step": (C.c_int, [_P, _P, C.POINTER(moe_weights), _P, C.POINTER(C.c_int32), _P, C.c_size_t, _P]),
+    "moe_stack_decode_step_trace": (C.c_int, [_P, _P, C.POINTER(moe_weights), _P, C.POINTER(C.c_int32), _P, C.c_size_t,
+                                              _P]),
     "moe_expert_replacements": (C.c_int, [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P]),
 }
 EXPORTS = tuple(_SIGS)
@@ -234,6 +236,14 @@ def moe_stack_decode_step(off: int, ctx: int, routers, h, n_layers: int, k: int,
     _ok(_lib().moe_stack_decode_step(off, ctx, routers, _ptr(h), trace, _ptr(ws), ws.numel() * ws.element_size(),
                                      _stream(stream)), "moe_stack_decode_step")
     return [list(trace[l * k:(l + 1) * k]) for l in range(n_layers)]
+
+
+def moe_stack_decode_step_trace(off: int, ctx: int, routers, h, sel, ws, stream=None):
+    """sel: [n_layers][k] nested list of the experts every layer has to use."""
+    flat = [int(e) for row in sel for e in row]
+    arr = (C.c_int32 * len(flat))(*flat)
+    _ok(_lib().moe_stack_decode_step_trace(off, ctx, routers, _ptr(h), arr, _ptr(ws), ws.numel() * ws.element_size(),
+                                           _stream(stream)), "moe_stack_decode_step_trace")
 
 
 def moe_expert_replacements(topk_trace, B, T, k, n_experts, h_total_out, stream=None):

@@ -21,6 +21,8 @@ struct moe_offload {
   size_t slot_bytes;
   cudaStream_t copy_stream;
   cudaEvent_t ev_compute, ev_copy;
+  std::vector<cudaEvent_t> layer_done;      // per layer: recorded after the layer's last kernel by the stacked steps
+  std::vector<char> layer_done_set;
   std::vector<std::vector<int>> recency;    // per layer: resident experts, least recently used first
   std::vector<std::vector<int>> slot_of;    // per layer: expert -> slot or -1
   int32_t* d_tables;                        // device [n_layers][E]
@@ -33,6 +35,22 @@ namespace cosmoe {
 namespace {
 
 constexpr size_t kCopyChunk = 8u << 20;  // host->device copies are issued in chunks of this size
+
+// A prescribed expert set for one token: the gate weights are the router's probabilities of those experts,
+// renormalised over the set (what the layer computes when it is told which experts to use).
+struct ForcedSel {
+  int32_t e[MOE_MAX_TOPK];
+};
+__global__ void forced_routing_kernel(const float* __restrict__ probs, int k, int renorm, ForcedSel f,
+                                      int32_t* __restrict__ idx, float* __restrict__ wt) {
+  const int lane = threadIdx.x;
+  const float p = lane < k ? probs[f.e[lane]] : 0.f;
+  const float sum = warp_sum(p);
+  if (lane < k) {
+    idx[lane] = f.e[lane];
+    wt[lane] = renorm ? p / sum : p;
+  }
+}
 
 // u = h / sqrt(mean(h^2)) -> x (bf16 or fp32); one CTA
 __global__ void rms_glue_kernel(const float* __restrict__ h, int d, void* __restrict__ x, int x_is_bf16) {
@@ -114,6 +132,12 @@ int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_pe
   if (e == cudaSuccess) e = cudaMallocHost((void**)&o->h_tables, tb);
   if (e == cudaSuccess) e = cudaMallocHost((void**)&o->h_route, sizeof(int32_t) * MOE_MAX_TOPK);
   if (e == cudaSuccess) {
+    o->layer_done.assign(n_layers, nullptr);
+    o->layer_done_set.assign(n_layers, 0);
+    for (int l = 0; l < n_layers && e == cudaSuccess; ++l)
+      e = cudaEventCreateWithFlags(&o->layer_done[l], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) {
     o->recency.assign(n_layers, std::vector<int>());
     o->slot_of.assign(n_layers, std::vector<int>(o->E, -1));
     for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
@@ -146,6 +170,8 @@ int moe_offload_destroy(moe_offload* o) {
   }
   if (o->ev_compute) cudaEventDestroy(o->ev_compute);
   if (o->ev_copy) cudaEventDestroy(o->ev_copy);
+  for (cudaEvent_t ev : o->layer_done)
+    if (ev) cudaEventDestroy(ev);
   if (o->d_tables) cudaFree(o->d_tables);
   if (o->h_tables) cudaFreeHost(o->h_tables);
   if (o->h_route) cudaFreeHost(o->h_route);
@@ -154,7 +180,9 @@ int moe_offload_destroy(moe_offload* o) {
   return MOE_OK;
 }
 
-int moe_offload_ensure(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, void* compute_stream) {
+// by_layer_event: the caller is a stacked step, which records layer_done[layer] after the layer's kernels
+static int ensure_impl(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, void* compute_stream,
+                       bool by_layer_event) {
   if (!o || !sel || layer < 0 || layer >= o->n_layers || n <= 0 || n > o->slots) return MOE_ERR_INVALID_ARG;
   for (int i = 0; i < n; ++i) {
     if (sel[i] < 0 || sel[i] >= o->E) return MOE_ERR_INVALID_ARG;
@@ -186,8 +214,14 @@ int moe_offload_ensure(moe_offload* o, int32_t layer, const int32_t* sel, int32_
     }
     if (victim < 0) return MOE_ERR_STATE;
     if (!waited) {  // work already queued on the compute stream may still read the victim's slot
-      MOE_CUDA_TRY(cudaEventRecord(o->ev_compute, cs));
-      MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->ev_compute, 0));
+      if (by_layer_event && o->layer_done_set[layer]) {
+        // the stacked steps record when a layer's kernels are done: only those read this layer's slots, so the
+        // copy need not wait for the other layers' kernels queued since
+        MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->layer_done[layer], 0));
+      } else {
+        MOE_CUDA_TRY(cudaEventRecord(o->ev_compute, cs));
+        MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->ev_compute, 0));
+      }
       waited = true;
     }
     const int slot = slot_of[victim];
@@ -214,6 +248,10 @@ int moe_offload_ensure(moe_offload* o, int32_t layer, const int32_t* sel, int32_
     MOE_CUDA_TRY(cudaStreamWaitEvent(cs, o->ev_copy, 0));
   }
   return MOE_OK;
+}
+
+int moe_offload_ensure(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, void* compute_stream) {
+  return ensure_impl(o, layer, sel, n, compute_stream, false);
 }
 
 int moe_offload_slot_table(moe_offload* o, int32_t layer, const int32_t** table) {
@@ -267,17 +305,68 @@ int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* route
     for (int j = 0; j < k; ++j) {
       if (trace_host) trace_host[(size_t)l * k + j] = o->h_route[j];
     }
-    rc = moe_offload_ensure(o, l, o->h_route, k, stream);
+    rc = ensure_impl(o, l, o->h_route, k, stream, true);
     if (rc != MOE_OK) return rc;
     moe_weights w = routers[l];
     w.gud = o->device_slots + (size_t)l * o->slots * o->slot_bytes;
     w.expert_slot = o->d_tables + (size_t)l * o->E;
     rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, y, nullptr, s);
     if (rc != MOE_OK) return rc;
+    MOE_CUDA_TRY(cudaEventRecord(o->layer_done[l], s));
+    o->layer_done_set[l] = 1;
     residual_kernel<<<(d + 255) / 256, 256, 0, s>>>(h, y, d, xbf);
     MOE_CUDA_TRY(cudaGetLastError());
     ctx->launches++;
   }
+  return MOE_OK;
+}
+
+int moe_stack_decode_step_trace(moe_offload* o, moe_ctx* ctx, const moe_weights* routers, float* h,
+                                const int32_t* sel_host, void* ws, size_t ws_bytes, void* stream) {
+  if (!o || !ctx || !routers || !h || !ws || !sel_host) return MOE_ERR_INVALID_ARG;
+  const moe_config& c = ctx->cfg;
+  if (c.wd_rank != 0 || c.d_model != o->cfg.d_model || c.d_ff != o->cfg.d_ff || c.n_experts != o->E ||
+      c.top_k != o->cfg.top_k)
+    return MOE_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(c, 1);
+  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
+  if ((size_t)c.d_ff * c.top_k * 2 < (size_t)c.d_model * 4 || (size_t)c.d_model * 2 < (size_t)c.n_experts * 4)
+    return MOE_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)stream;
+  char* wsb = (char*)ws;
+  int32_t* idx = (int32_t*)(wsb + L.topk_idx);
+  float* wt = (float*)(wsb + L.topk_w);
+  void* u = wsb + L.hidden;
+  void* y = wsb + L.out_slots;
+  float* probs = (float*)(wsb + L.xperm);  // [E] fp32; the region holds d bf16 values
+  const int d = c.d_model, k = c.top_k;
+  const int xbf = c.x_dtype == MOE_BF16;
+  for (int l = 0; l < o->n_layers; ++l) {
+    ForcedSel f{};
+    for (int j = 0; j < k; ++j) f.e[j] = sel_host[(size_t)l * k + j];
+    // the copies of this layer's misses are queued before its kernels: they run on the copy stream while the
+    // compute stream is still busy with the layers before
+    int rc = ensure_impl(o, l, f.e, k, stream, true);
+    if (rc != MOE_OK) return rc;
+    rms_glue_kernel<<<1, 256, 0, s>>>(h, d, u, xbf);
+    MOE_CUDA_TRY(cudaGetLastError());
+    rc = launch_route(ctx, u, 1, &routers[l], idx, wt, probs, s);
+    if (rc != MOE_OK) return rc;
+    forced_routing_kernel<<<1, 32, 0, s>>>(probs, k, c.renorm, f, idx, wt);
+    MOE_CUDA_TRY(cudaGetLastError());
+    moe_weights w = routers[l];
+    w.gud = o->device_slots + (size_t)l * o->slots * o->slot_bytes;
+    w.expert_slot = o->d_tables + (size_t)l * o->E;
+    rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, y, nullptr, s);
+    if (rc != MOE_OK) return rc;
+    MOE_CUDA_TRY(cudaEventRecord(o->layer_done[l], s));
+    o->layer_done_set[l] = 1;
+    residual_kernel<<<(d + 255) / 256, 256, 0, s>>>(h, y, d, xbf);
+    MOE_CUDA_TRY(cudaGetLastError());
+    ctx->launches += 3;
+  }
+  // the per-layer staging of the slot tables is reused by the next step
+  MOE_CUDA_TRY(cudaStreamSynchronize(s));
   return MOE_OK;
 }
 

@@ -154,6 +154,10 @@ class OffloadedStack:
         """h: fp32 [d] device tensor, updated in place.  Returns the per-layer selections."""
         return B.moe_stack_decode_step(self.off, self.ctx, self.routers, h, self.n_layers, self.k, self.ws)
 
+    def step_trace(self, h, sel):
+        """The same step with every layer's expert set given (sel [n_layers][k]); no host wait between layers."""
+        B.moe_stack_decode_step_trace(self.off, self.ctx, self.routers, h, sel, self.ws)
+
     def stats(self):
         return B.moe_offload_stats(self.off)
 

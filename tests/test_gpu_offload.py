@@ -77,6 +77,51 @@ def test_stacked_decode_with_offload_matches_checker(slots):
     stack.close()
 
 
+@pytest.mark.parametrize("p_stay", [0.12, 0.87])
+def test_stacked_decode_with_prescribed_expert_sets(p_stay):
+    """Replay of sticky routing traces under the rule of Eq. 8 (capacity = k): outputs against the checker told to
+    use the same sets, traffic against the policy simulation, replacement ratio (Eq. 4-5) of the trace itself."""
+    sh = W.LayerShape("t", 5, 256, 512, n_experts=8, top_k=2, x_dtype="bf16", bias="none")
+    n_layers, steps, slots = 3, 12, 2
+    stack, host = make_stack(sh, n_layers, slots)
+    traces = [W.sticky_routing_trace(777 + l, steps, sh.n_experts, sh.top_k, p_stay).tolist() for l in range(n_layers)]
+    for step in range(steps):
+        h0 = W.make_x(sh.with_(x_dtype="f32"), 1, device="cuda", step=step)[0].contiguous()
+        h = h0.clone()
+        sel = [traces[l][step] for l in range(n_layers)]
+        stack.step_trace(h, sel)
+        torch.cuda.synchronize()
+        assert stack.check() == 0
+        hh = h0.cpu().numpy().astype(np.float64)
+        for l in range(n_layers):
+            u = O.rms_glue(hh[None])[0]
+            u_b = torch.from_numpy(u.astype(np.float32)).to(torch.bfloat16)
+            ex = {k: v for k, v in host[l].items() if k not in ("w_router", "b_router")}
+            ora = O.layer_forward(W.to_host_bits(u_b[None]), host[l]["w_router"], host[l]["b_router"], ex, sh.top_k,
+                                  forced_topk=np.int32([sel[l]]))
+            hh = hh + torch.from_numpy(ora["y"][0].astype(np.float32)).to(torch.bfloat16).double().numpy()
+        U.assert_close_rms(h.cpu().numpy().astype(np.float64), hh, tol=U.Y_TOL, what=f"h after step {step}")
+    st = stack.stats()
+    tot = {"n_fetch": 0, "bytes": 0, "hits": 0}
+    for l in range(n_layers):
+        sim = F.lru_cache_sim(traces[l], sh.n_experts, slots, stack.slot_bytes)
+        for k in tot:
+            tot[k] += sim[k]
+        assert stack.resident(l) == sim["slots"][-1]
+        eq8 = F.eq8_policy(traces[l])
+        assert [sorted(e for e, _ in f) for f in sim["fetches"]][1:] == eq8[1:]
+    assert (st["fetches"], st["bytes"], st["hits"]) == (tot["n_fetch"], tot["bytes"], tot["hits"])
+    # the device-side metric on the same traces
+    tr = torch.tensor(traces, dtype=torch.int32, device="cuda")
+    hsum = torch.zeros(1, dtype=torch.int64, device="cuda")
+    from paper_2503_00245_b200 import binding as B
+    B.moe_expert_replacements(tr, n_layers, steps, sh.top_k, sh.n_experts, hsum)
+    torch.cuda.synchronize()
+    want = sum(X.hard_replacements(X.activity_from_topk(np.int32(traces[l])[None], sh.n_experts))[1] for l in range(n_layers))
+    assert int(hsum.item()) == want
+    stack.close()
+
+
 def test_offload_ensure_argument_errors():
     from paper_2503_00245_b200 import binding as B
     sh = W.LayerShape("t", 5, 256, 512, n_experts=8, top_k=2)
