@@ -670,11 +670,13 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   }
   // the router's weights do not depend on any earlier kernel: the first group of eight experts is fetched
   // before the dependency wait, so its DRAM latency overlaps the predecessor's tail
-  uint4 wr0[kXIters];
+  // (input features per thread in the router: 4 cover d <= 1024, the shapes of these variants)
+  constexpr int kRJ = (V == V_T1 || V == V_MMA_BF16_S || V == V_MMA_F32_S) ? 4 : kXIters;
+  uint4 wr0[kRJ];
   const bool prefetched = P.fused_route && warp < kWarps && (P.E & 7) == 0;
   if (prefetched) {
 #pragma unroll
-    for (int j = 0; j < kXIters; ++j)
+    for (int j = 0; j < kRJ; ++j)
       wr0[j] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + j * kConsumerThreads, P.d - 1) * P.E));
   }
   if (tid != kConsumerThreads) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -685,17 +687,17 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       const int d = P.d, E = P.E;
       if ((E & 7) == 0) {
         // this thread's input features (d <= 2048: at most 8), fetched in one round trip
-        float xv[kXIters];
+        float xv[kRJ];
 #pragma unroll
-        for (int j = 0; j < kXIters; ++j) {
+        for (int j = 0; j < kRJ; ++j) {
           const int i = min(tid + j * kConsumerThreads, d - 1);
           xv[j] = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[i]) : ((const float*)P.x)[i];
           if (tid + j * kConsumerThreads >= d) xv[j] = 0.f;
         }
         for (int e8 = 0; e8 < E; e8 += 8) {
-          uint4 wr[kXIters];
+          uint4 wr[kRJ];
 #pragma unroll
-          for (int j = 0; j < kXIters; ++j)
+          for (int j = 0; j < kRJ; ++j)
             wr[j] = e8 == 0 ? wr0[j]
                             : __ldg(reinterpret_cast<const uint4*>(P.w_router +
                                                                    (size_t)min(tid + j * kConsumerThreads, d - 1) * E + e8));
@@ -703,7 +705,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
 #pragma unroll
           for (int j = 0; j < 8; ++j) a[j] = 0.f;
 #pragma unroll
-          for (int j = 0; j < kXIters; ++j) {
+          for (int j = 0; j < kRJ; ++j) {
             float w[8];
             unpack8(wr[j], w);
 #pragma unroll
