@@ -105,8 +105,11 @@ __device__ __forceinline__ void item_bounds(const Smem& sm, int f, PassIt& g) {
   g.ngrp = (ne + kMaxN - 1) / kMaxN;
   g.grp = 0;
 }
-__device__ __forceinline__ void pass_init(const Smem& sm, int f, PassIt& g) {
-  const unsigned G = gridDim.x, b = blockIdx.x, na = (unsigned)sm.n_act;
+// This CTA's share [u0, u1) of the na * f hidden units of the active experts: a function of the launch shape and
+// of the NUMBER of active experts only (a single token always has k of them, so its share can be worked out
+// before the routing is known -- the divisions below then leave the launch's serial path).
+__device__ __forceinline__ void pass_split(unsigned na, int f, PassIt& g) {
+  const unsigned G = gridDim.x, b = blockIdx.x;
   g.ra = g.rb = g.grp = g.ngrp = 0;
   if (na > 0 && na <= 16u && G >= na) {
     // few active experts: every CTA works for ONE expert (a second pass costs its set-up and its output atomics
@@ -129,11 +132,16 @@ __device__ __forceinline__ void pass_init(const Smem& sm, int f, PassIt& g) {
   if (g.u1 > g.u0) {
     g.ai = (int)((unsigned)g.u0 / (unsigned)f);
     g.ai_hi = (int)((unsigned)(g.u1 - 1) / (unsigned)f);
-    item_bounds(sm, f, g);
   } else {
     g.ai = 0;
     g.ai_hi = -1;
   }
+}
+// `presplit`: pass_split(hint_na) has already filled g; it stands if the routing found that many active experts.
+__device__ __forceinline__ void pass_init(const Smem& sm, int f, PassIt& g, bool presplit = false, unsigned hint_na = 0u) {
+  const unsigned na = (unsigned)sm.n_act;
+  if (!presplit || na != hint_na) pass_split(na, f, g);
+  if (g.ai <= g.ai_hi) item_bounds(sm, f, g);
 }
 __device__ __forceinline__ bool next_pass(const Smem& sm, int f, PassIt& g, Pass& ps) {
   for (;;) {
@@ -668,6 +676,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       bulk_g2s(xs, P.x, bytes, &sm.xfull[0]);
     }
   }
+  PassIt pit;
+  if (fused1) pass_split((unsigned)P.k, P.f, pit);  // a single token has k active experts: known before the routing
   // the router's weights do not depend on any earlier kernel: the first group of eight experts is fetched
   // before the dependency wait, so its DRAM latency overlaps the predecessor's tail
   // (input features per thread in the router: 4 cover d <= 1024, the shapes of these variants)
@@ -953,8 +963,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   }
   __syncthreads();
 
-  PassIt pit;
-  pass_init(sm, P.f, pit);
+  pass_init(sm, P.f, pit, fused1, (unsigned)P.k);
   Pass ps;
   RingPos rp{0, 0u, 0};
 
@@ -1074,7 +1083,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   // CTAs they wait for are running or can start on the SMs the finished ones have left.
   const unsigned G = gridDim.x, K = G < (unsigned)kFinalizers ? G : (unsigned)kFinalizers;
   if (tid == 0) {
-    __threadfence();
+    // (the barrier above orders every warp's accumulator atomics before this thread; the arrival below is a
+    // release at GPU scope, so they are performed before the count moves -- no separate fence)
     const unsigned long long old_total = atom_add_acq_rel64(&st->done_total, 1ull);
     const unsigned old = (unsigned)(old_total % G);  // this CTA's arrival number within the launch
     const unsigned long long target = old_total - old + G;
@@ -1089,8 +1099,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
       }
     }
-    sm.last = slice;
-    __threadfence();
+    sm.last = slice;  // (published to the CTA by the barrier below; the counter was read with acquire loads)
   }
   fin = consumer_sync(sm, cpar, lane) && fin;
   const int slice = sm.last;

@@ -504,12 +504,11 @@ __global__ void __launch_bounds__(kThreads, 1) stream_ffn_kernel(const StreamPar
         __syncwarp();
         int okb = 1;
         if (lane == 0) {
+          // (release / acquire at GPU scope on the counter and the generation word order the stores: no fences)
           const unsigned gen0 = ld_acquire(&P.st->bar_gen);
-          __threadfence();
           const unsigned old = atom_add_acq_rel(&P.st->bar_count, 1u);
           if (old == gridDim.x - 1u) {
             P.st->bar_count = 0u;
-            __threadfence();
             st_release(&P.st->bar_gen, gen0 + 1u);
           } else {
             const long long t0 = clock64();
@@ -522,7 +521,6 @@ __global__ void __launch_bounds__(kThreads, 1) stream_ffn_kernel(const StreamPar
               }
             }
           }
-          __threadfence();
         }
         okb = __shfl_sync(0xffffffffu, okb, 0);
         if (!okb) {

@@ -58,7 +58,8 @@ __device__ __forceinline__ bool meet(DeviceState* st, WdSmem& sm) {
   __syncthreads();
   if (threadIdx.x == 0) {
     const unsigned G = gridDim.x;
-    __threadfence();
+    // (the arrival is a release at GPU scope and the barrier above orders the CTA's stores before it; the wait
+    // reads the counter with acquire loads: no separate fences)
     const unsigned long long old = atom_add_acq_rel64(&st->phase_total, 1ull);
     const unsigned long long target = old - old % G + G;
     int ok = 1;
@@ -70,7 +71,6 @@ __device__ __forceinline__ bool meet(DeviceState* st, WdSmem& sm) {
         break;
       }
     }
-    __threadfence();
     sm.ok = ok;
   }
   __syncthreads();
