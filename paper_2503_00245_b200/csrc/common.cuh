@@ -312,17 +312,27 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
 
+// fp32 -> unsigned key with the same order (-0 counts as +0; NaN is not ordered), and back
+__device__ __forceinline__ unsigned f32_key(float v) {
+  const unsigned b = __float_as_uint(v + 0.0f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float f32_unkey(unsigned k) {
+  return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
+}
+
 // Softmax over E logits (Eq. 2), top-k (Eq. 3) and gate weights by one warp: lane l holds logit l (l0)
 // and logit l + 32 (l1).  Selection runs on the logits (softmax is monotonic, and the logits carry more
 // bits than fp32 probabilities); ties go to the lower expert index.  Lane j < k writes the j-th choice.
+// (maxima go through the warp's integer reduction, one instruction instead of five shuffle rounds: this
+// routine sits on the serial path of every decode launch)
 __device__ __forceinline__ void warp_route_finish(float l0, float l1, int E, int k, int renorm, int lane,
                                                   int32_t* __restrict__ idx_out, float* __restrict__ w_out,
                                                   float* __restrict__ probs_out) {
+  const unsigned FULL = 0xffffffffu;
   const float NEG = -3.402823466e38f;
   const bool has0 = lane < E, has1 = lane + 32 < E;
-  float m = fmaxf(has0 ? l0 : NEG, has1 ? l1 : NEG);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float m = f32_unkey(__reduce_max_sync(FULL, f32_key(fmaxf(has0 ? l0 : NEG, has1 ? l1 : NEG))));
   const float p0 = has0 ? expf(l0 - m) : 0.f, p1 = has1 ? expf(l1 - m) : 0.f;
   const float inv_sum = 1.0f / warp_sum(p0 + p1);
   if (probs_out) {
@@ -338,17 +348,14 @@ __device__ __forceinline__ void warp_route_finish(float l0, float l1, int E, int
     int id = 0x7fffffff;
     if (free0) v = l0, id = lane;
     if (free1 && (!free0 || l1 > v)) v = l1, id = lane + 32;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-      const int oid = __shfl_xor_sync(0xffffffffu, id, o);
-      if (ov > v || (ov == v && oid < id)) v = ov, id = oid;
-    }
-    if (id == lane) free0 = false;
-    if (id == lane + 32) free1 = false;
-    const float pw = expf(v - m) * inv_sum;
+    const unsigned key = id != 0x7fffffff ? f32_key(v) : 0u;
+    const unsigned best = __reduce_max_sync(FULL, key);
+    const int win = (int)__reduce_min_sync(FULL, (unsigned)((key == best) ? id : 0x7fffffff));
+    if (win == lane) free0 = false;
+    if (win == lane + 32) free1 = false;
+    const float pw = expf(f32_unkey(best) - m) * inv_sum;
     wtot += pw;
-    if (lane == j) my_w = pw, my_idx = id;
+    if (lane == j) my_w = pw, my_idx = win;
   }
   if (lane < k) {
     idx_out[lane] = my_idx;
