@@ -235,8 +235,8 @@ def _launches(r):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
 # under profiles/ (same workload, ring of fewer layers).  An entry is dropped when its kernel changes.
 NCU_TRAFFIC_BYTES = {
-    "wearable-decode-T1": 34_780_416,                    # dense_stream_kernel, one launch per step
-    "wearable-decode-T8": 121_373_696 + 3_687_424,       # dense_stream_kernel, launch with 7 active experts
+    "wearable-decode-T1": 34_782_976,                    # dense_stream_kernel, one launch per step
+    "wearable-decode-T8": 121_376_256 + 3_742_720,       # dense_stream_kernel, launch with 7 active experts
     "phone-prefill-T2048": 473_914_112 + 40_779_008,     # grouped_gemm_kernel, the first (larger) GEMM of the layer
 }
 
