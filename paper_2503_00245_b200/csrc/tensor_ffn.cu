@@ -531,17 +531,19 @@ int launch_gg(moe_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const 
   P.E = c.n_experts;
   P.st = ctx->d_state;
   const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
-  // 256-row tiles halve the operand traffic per flop; small problems keep 128-row tiles to fill the SMs
+  // 256-row tiles read every B slice once for up to 256 rows of an expert (half the operand traffic per flop,
+  // and an expert with 129..256 rows is one tile instead of two); problems whose 256-row tiles would leave SMs
+  // without work keep 128-row tiles.  A cut contraction (ksplit) multiplies the work items.
   P.tile_rows = kBM;
-  if (!P.dual_a && (long long)((n_slots + kTileRows - 1) / kTileRows) * n_tiles >= 2ll * ctx->sm_count)
-    P.tile_rows = kTileRows;
+  if (P.ksplit < 1) P.ksplit = 1;
+  const long long m256 = std::max<long long>((n_slots + kTileRows - 1) / kTileRows, std::min(c.n_experts, n_slots));
+  if (!P.dual_a && (m256 * n_tiles >= ctx->sm_count || P.ksplit > 1)) P.tile_rows = kTileRows;
   P.single_a = (P.tile_rows == kBM && !P.dual_a) ? 1 : 0;
   P.n_stages = P.single_a ? 4 : 3;
   const size_t stage_bytes = (size_t)kBM * kBK * 2 * (P.single_a ? 1 : 2) + 256 * kBK * 2;
   const size_t smem = P.n_stages * stage_bytes + sizeof(SmemGG) + 1024 + 128;
   if ((long long)smem > ctx->max_smem_optin) return MOE_ERR_UNSUPPORTED;
   const long long m_tiles = (n_slots + P.tile_rows - 1) / P.tile_rows + c.n_experts;  // upper bound
-  if (P.ksplit < 1) P.ksplit = 1;
   const int grid = (int)std::min<long long>(m_tiles * n_tiles * P.ksplit, ctx->sm_count);
   MOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   MOE_CUDA_TRY(launch_pdl(grouped_gemm_kernel, dim3(grid), dim3(kThreadsGG), smem, s, a0, a1, b, P));
