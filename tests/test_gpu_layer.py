@@ -115,6 +115,28 @@ def test_back_to_back_calls_with_different_inputs(T):
         U.assert_close_rms(U.to64(y), ora["y"])
 
 
+@pytest.mark.parametrize("sh,T", [(W.WEARABLE, 1), (W.WEARABLE, 8), (W.PHONE, 1), (W.PHONE_WD128, 1), (W.PHONE_WD1024, 1)])
+def test_long_run_of_queued_calls_is_bitwise_stable(sh, T):
+    """Two thousand launches queued back to back, alternating four inputs, each output kept: every output must
+    equal, bit for bit, the first one its input produced.  The fixed-point partial sums, the arrival counter that
+    runs over launches and the finalisers' reads are ordered only by release/acquire operations; a launch that
+    finalised before a neighbour's (or its own) sums had landed would show here."""
+    lay, t, host = U.build(sh, T, path=STREAM)
+    xs = [W.make_x(sh, T, device="cuda", step=s) for s in range(4)]
+    first = [lay.forward(x).clone() for x in xs]
+    torch.cuda.synchronize()
+    n = 2000
+    out = torch.empty((n,) + tuple(first[0].shape), dtype=first[0].dtype, device="cuda")
+    for i in range(n):
+        lay.forward(xs[i % 4], y=out[i])
+    torch.cuda.synchronize()
+    assert lay.check() == 0
+    for j in range(4):
+        same = (out[j::4].view(torch.int16 if out.dtype == torch.bfloat16 else torch.int32)
+                == first[j].view(torch.int16 if out.dtype == torch.bfloat16 else torch.int32))
+        assert bool(same.all()), f"input {j}: {int((~same).sum())} differing elements over {n // 4} launches"
+
+
 def O_near(ora, k):
     from oracle import moe_oracle as O
     return O.near_tie_tokens(ora["logits"], k, U.TIE_GAP)
