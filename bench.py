@@ -238,6 +238,9 @@ NCU_TRAFFIC_BYTES = {
     "wearable-decode-T1": 34_782_976,                    # dense_stream_kernel, one launch per step
     "wearable-decode-T8": 121_376_256 + 3_742_720,       # dense_stream_kernel, launch with 7 active experts
     "phone-prefill-T2048": 473_914_112 + 40_779_008,     # grouped_gemm_kernel, the first (larger) GEMM of the layer
+    "phone-decode-T1": 138_686_976 + 3_785_472,          # dense_stream_kernel
+    "phone-wd128-decode-T1": 11_899_904,                 # wd_decode_kernel
+    "phone-wd1024-decode-T1": 94_490_624 + 3_387_392,    # stream_ffn_kernel
 }
 
 
