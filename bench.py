@@ -250,6 +250,14 @@ def roofline(res):
     return r
 
 
+def _decode_kernel_name(shape, T):
+    """The kernel that streams the experts at this shape (the library's dispatch rule, restated for the label)."""
+    if not shape.wd_rank:
+        return "dense_stream_kernel"
+    wd_bytes = shape.top_k * W.expert_bytes(shape)
+    return "wd_decode_kernel" if (T == 1 and wd_bytes <= 32 * 1024 * 1024) else "stream_ffn_kernel"
+
+
 def _roofline(res):
     shape, T, pk = res["shape"], res["T"], res["peaks"]
     sec = res["ms_per_step"] * 1e-3
@@ -258,7 +266,7 @@ def _roofline(res):
         ach = b / sec / 1e9
         return {"bound": "hbm", "achieved": round(ach, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": round(ach / pk["hbm_gbs"], 4), "traffic": None, "peak_source": pk["source"],
-                "bytes_per_launch": int(b), "kernel": "dense_stream_kernel",
+                "bytes_per_launch": int(b), "kernel": _decode_kernel_name(shape, T),
                 "note": "duration = whole step (router + expert kernel) / 1"}
     fl = flops(shape, T)
     t_tc = fl / (pk["tflops_sustained"] * 1e12)
