@@ -42,8 +42,9 @@ WsLayout ws_layout(const moe_config& c, int T) {
   L.vec_c = take(stream_ok ? n * (size_t)c.wd_rank * 8 * 4 : 0);  // v, in up to 8 segments per value
   L.xperm = take(tensor_ok ? n * (size_t)c.d_model * 2 : 0);
   L.hidden = take(tensor_ok ? n * (size_t)c.d_ff * 2 : 0);
-  L.mid_a = take(tensor_ok ? n * 4 * (size_t)c.wd_rank * 2 : 0);  // t_g, t_u as hi + lo bf16 pairs
-  L.mid_b = take(tensor_ok ? n * 2 * (size_t)c.wd_rank * 2 : 0);  // v as a hi + lo pair
+  const size_t rp = ((size_t)c.wd_rank + 63) / 64 * 64;            // the rank rounded up to the tensor path's K step
+  L.mid_a = take(tensor_ok ? n * 4 * rp * 2 : 0);  // t_g, t_u as hi + lo bf16 pairs
+  L.mid_b = take(tensor_ok ? n * 2 * rp * 2 : 0);  // v as a hi + lo pair
   L.out_slots = take(n * (size_t)c.d_model * 4 * (n <= (size_t)kKSplitMaxSlots ? kKSplitMax : 1));  // room for partial-sum planes
   L.total = off + A;
   return L;
@@ -51,7 +52,9 @@ WsLayout ws_layout(const moe_config& c, int T) {
 
 static int pick_path(const moe_config& c, int T) {
   if (c.path != MOE_PATH_AUTO) return c.path;
-  return T <= MOE_STREAM_MAX_TOKENS ? MOE_PATH_STREAM : MOE_PATH_TENSOR;
+  if (T > MOE_STREAM_MAX_TOKENS) return MOE_PATH_TENSOR;
+  if (c.wd_rank == 0 && c.d_model > kDenseStreamMaxD) return MOE_PATH_TENSOR;  // the tensor path takes any width
+  return MOE_PATH_STREAM;
 }
 
 static bool misaligned(const void* p) { return ((uintptr_t)p & 15u) != 0; }
@@ -129,7 +132,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out) {
   c->d_state = nullptr;
   c->h_state = nullptr;
   c->acc = nullptr;
-  c->acc_elems = (cfg->wd_rank == 0 && cfg->d_model <= 2048)
+  c->acc_elems = (cfg->wd_rank == 0 && cfg->d_model <= kDenseStreamMaxD)
                      ? (size_t)MOE_STREAM_MAX_TOKENS * cfg->top_k * cfg->d_model
                      : 0;
   cudaError_t e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);

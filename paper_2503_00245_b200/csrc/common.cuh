@@ -76,6 +76,7 @@ int launch_route(moe_ctx* ctx, const void* x, int T, const moe_weights* w, int32
 int launch_permute(moe_ctx* ctx, const int32_t* idx, int T, int32_t* offsets, int32_t* perm, int32_t* inv,
                    cudaStream_t s);
 // out_slots may come as `planes` partial sums, one [T*k][d] plane after the other (summed in order).
+constexpr int kDenseStreamMaxD = 2048;  // widest d_model the dense streaming kernel handles (token row in registers)
 constexpr int kKSplitMax = 4;          // planes the tensor path may ask for ...
 constexpr int kKSplitMaxSlots = 2048;  // ... when there are at most this many (token, choice) slots
 int launch_combine(moe_ctx* ctx, const float* out_slots, const float* wt, const int32_t* inv, int T, void* y,

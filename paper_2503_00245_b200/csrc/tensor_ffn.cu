@@ -7,16 +7,24 @@
 //                  (2) O = H Wd                  A = H,           B = down rows of gud (N-major) -> fp32 slots
 //   Eq. 1 factors  (1) T = X [gL | uL]   (2) H = silu(Tg gR) * (Tu uR)   (3) V = H dL   (4) O = V dR
 //
-// One CTA computes one tile of up to 256 rows x 256 columns: two 128-row halves with their own accumulators
-// share every B slice (128 flop per operand byte moved from L2, against 85 for a 128-row tile); a tile whose
-// second half would be empty (the ragged end of an expert's rows) runs one half.  Roles:
+// Two CTAs on neighbouring SMs (a cluster of 2) compute one tile of 256 rows x up to 256 columns with
+// tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of A and HALF of the tile's B rows, the tensor
+// cores of the pair exchange the B halves, and each CTA ends up with the accumulators of its 128 rows
+// (128 TMEM lanes x N columns).  Per flop a CTA moves half the B bytes into shared memory and reads a third
+// fewer operand bytes out of it than a single CTA computing 256 x 256 on its own, and the tile takes 256 of the
+// 512 TMEM columns, so the accumulators are double-buffered: the epilogue of tile i runs under the MMAs of
+// tile i + 1.  Roles in each CTA:
 //   warp 0     TMA producer: 64-wide K slices of A and B into a ring of shared-memory stages (128-byte swizzle);
-//   warp 1     allocates tensor memory and issues tcgen05.mma (M = 128, N <= 256, K = 16 per instruction) with
-//              fp32 accumulators in TMEM; a commit releases each stage back to the producer;
-//   warps 2-5  epilogue: tcgen05.ld the accumulators (one TMEM lane = one output row per thread), apply
+//              both CTAs' copies complete on the LEADER's (rank 0) stage barrier;
+//   warp 1     allocates tensor memory (both CTAs); in the leader one thread issues the MMAs for the pair
+//              (M = 256, N <= 256, K = 16 per instruction) and commits to both CTAs' barriers;
+//   warps 2-9  epilogue: tcgen05.ld the accumulators (one TMEM lane = one output row per thread), apply
 //              SiLU * mul or nothing, convert, store the rows that belong to the expert.
+// Tiles are handed out statically (pair p takes tiles p, p + pairs, ...): both CTAs of a pair derive the same
+// sequence without talking to each other.
 // Ragged groups: a tile may read rows of the next expert (or zeros past the end); they are never stored.
 // K and N tails are zero-filled by TMA.  All waits are bounded; an expired wait sets the ctx's status word.
+// No copy in this file uses cluster multicast: every CTA fetches what it needs with its own loads.
 #include <cuda.h>
 
 #include <algorithm>
@@ -27,28 +35,34 @@ namespace cosmoe {
 
 namespace {
 
-constexpr int kBM = 128;  // rows per tile (TMEM lanes)
+constexpr int kBM = 128;  // rows per CTA and tile (TMEM lanes)
 constexpr int kBK = 64;   // K elements per stage (128 bytes of bf16 = one swizzle row)
-constexpr int kTileQueue = 8;  // tile indices in flight between the producer and the other roles
 constexpr int kEpiWarps = 8;  // two per quarter of the TMEM lanes, splitting the columns
 constexpr int kThreadsGG = (2 + kEpiWarps) * 32;
-constexpr int kTmemCols = 512;  // two accumulators of 256 columns
-constexpr int kMaxStagesGG = 4;
-constexpr int kTileRows = 2 * kBM;  // rows per tile when the A operand is single (two halves)
+constexpr int kTmemCols = 512;  // two accumulator buffers of 256 columns
+constexpr int kAccCols = 256;
+constexpr int kMaxStagesGG = 6;
+constexpr int kPairRows = 2 * kBM;  // rows of a pair's tile
 
 enum Epi { EPI_SWIGLU = 0, EPI_BF16_PAIR = 1, EPI_BF16 = 2, EPI_F32 = 3 };
+// How the B operand of a tile is laid out and shared between the two CTAs of a pair (rank 0 / rank 1):
+enum BMode {
+  B_PAIR = 0,    // interleaved matrix, columns [0, bn) = sub-row 0 (rank 0 loads them), [bn, 2 bn) = sub-row 1 (rank 1)
+  B_DUAL = 1,    // the same columns, but sub-row 1 meets a second A operand: two MMAs of N = bn, each rank loads half of both
+  B_SINGLE = 2,  // one sub-row, K-major: rank r loads rows [n0 + r bn/2, n0 + (r+1) bn/2)
+  B_NMAJOR = 3   // one sub-row stored [k][n] (the down rows of gud): rank r loads its bn/2 columns in 64-column boxes
+};
 
 struct GGParams {
   const int32_t* offsets;  // [E+1] slot ranges per expert
   int E;
   int K;         // contraction length
-  int n_total;   // output columns (per half when `pair`)
-  int bn;        // output columns per tile (per half when `pair`): <= 128 when pair, <= 256 otherwise
-  int pair;      // B tile = two halves (sub-rows 0 and 1 of an interleaved matrix): accumulator columns [0,bn) and [128,128+bn)
-  int dual_a;    // the second half has its own A operand
-  int b_nmajor;  // B is stored [k][n] (n contiguous): the down rows of gud
-  int b_sub;     // sub-row of the interleaved matrix that single / N-major tiles read
-  int tile_rows; // rows per tile: 256 (two halves) or 128
+  int n_total;   // output columns (per sub-row in B_PAIR / B_DUAL)
+  int n_store;   // columns stored, >= n_total: the columns between are written as zeros (accumulators of B rows that do
+                 // not exist), so that a consumer may read the padded width
+  int bn;        // output columns per tile (per sub-row in B_PAIR / B_DUAL: <= 128; else <= 256)
+  int bmode;
+  int b_sub;     // sub-row of the interleaved matrix that B_SINGLE / B_NMAJOR tiles read
   int k_wrap;    // > 0: the B operand's k coordinate wraps at k_wrap (A = [hi | lo] halves of a split operand)
   int split;     // bf16 epilogues also store the rounding remainder: value = hi + lo, lo at column offset out_off_lo
   int epi;
@@ -56,8 +70,7 @@ struct GGParams {
   long long ld_out;    // elements
   long long out_off2;  // EPI_BF16_PAIR: column offset of the second half
   long long out_off_lo;  // split: column offset of the remainders
-  int ctr_idx;            // which word of DeviceState::tile_ctr hands out this launch's tiles (the other is cleared)
-  int single_a;           // 128-row tiles, one A operand: the stage has no A' part
+  int tail_split;         // B_NMAJOR, bn = 256: the tiles of the last, partly filled round are cut into two 128-column halves
   int ksplit;             // the contraction is cut into this many parts, each a work item of its own ...
   long long plane_elems;  // ... writing its partial sums plane_elems further on in `out` (EPI_F32 only)
   int n_stages;
@@ -65,33 +78,57 @@ struct GGParams {
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------------------
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+// Tiled loads whose completion may be counted on a barrier of the other CTA of the pair (cta_group::2); the
+// data always lands in the issuing CTA's own shared memory.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
-          "r"(smem_u32(dst)),
-      "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], "
+      "[%4];" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                            uint64_t* bar) {
+                                            uint32_t bar_cluster) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], "
-      "[%6];" ::"r"(smem_u32(dst)),
-      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, "
+      "%5}], [%6];" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar_cluster)
       : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory object in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_rank(const void* smem_ptr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(smem_ptr)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+// The barrier at this shared-memory offset gets one arrival IN BOTH CTAs of the pair when every MMA this thread
+// has issued so far has completed.  (A multicast of barrier arrivals, not of data: no copy in this file is multicast.)
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                   smem_u32(bar)),
+               "h"((unsigned short)3)
                : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool acc) {
+// `acc` == 0: the product overwrites the accumulator; otherwise it is added.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)acc)
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* v) {
@@ -111,6 +148,8 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 // Shared-memory operand descriptor (128-byte swizzle).  K-major tiles: rows of 128 bytes, 8-row groups 1024
 // bytes apart (stride byte offset), the leading offset is not used.  N-major tiles: 64 columns (128 bytes) per
 // k-row, 8-k-row groups 1024 bytes apart (stride), 64-column blocks `lbo` bytes apart (leading).
+// The start address sits in the low 14 bits (in units of 16 bytes), so stepping through a stage or through the
+// ring is an addition to the low word.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   uint64_t d = 0;
   d |= (uint64_t)((addr & 0x3ffffu) >> 4);
@@ -120,7 +159,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   d |= 2ull << 61;  // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K- or N-major, M = 128, N = n.
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K- or N-major, M = 256 over the pair, N = n.
 __device__ __forceinline__ uint32_t instr_desc(int n, bool b_nmajor) {
   uint32_t d = 0;
   d |= 1u << 4;   // accumulator format: fp32
@@ -128,66 +167,75 @@ __device__ __forceinline__ uint32_t instr_desc(int n, bool b_nmajor) {
   d |= 1u << 10;  // B: bf16
   d |= (b_nmajor ? 1u : 0u) << 16;
   d |= (uint32_t)(n >> 3) << 17;
-  d |= (uint32_t)(kBM >> 4) << 24;
+  d |= (uint32_t)(kPairRows >> 4) << 24;
   return d;
 }
 
 struct SmemGG {
-  uint64_t full[kMaxStagesGG];
-  uint64_t empty[kMaxStagesGG];
-  uint64_t accum_full;   // all MMAs of the current tile have completed
-  uint64_t accum_empty;  // the epilogue has read the accumulators out of TMEM (all epilogue warps arrive)
-  uint64_t tq_full[kTileQueue];   // the producer has put a tile index into tq[i]
-  uint64_t tq_empty[kTileQueue];  // the MMA thread and every epilogue warp have read it
-  int tq[kTileQueue];
+  uint64_t full[kMaxStagesGG];   // leader's: both CTAs' operands of the stage have landed
+  uint64_t empty[kMaxStagesGG];  // own: the MMAs have finished reading this CTA's stage
+  uint64_t accum_full[2];        // own: all MMAs of the tile in accumulator buffer b have completed
+  uint64_t accum_empty[2];       // leader's: the epilogue warps of both CTAs have read buffer b out of TMEM
   uint32_t tmem_base;
   int abort;
-  int tile_prefix[MOE_MAX_EXPERTS + 1];  // row tiles per expert, exclusive scan
+  int tile_prefix[MOE_MAX_EXPERTS + 1];  // 256-row tiles per expert, exclusive scan
 };
 
 struct Tile {
-  int e, m0, m_end, halves, n0, ks;
+  int e, m0, m_end, n0, ks, bn;
 };
 
-// idx-th tile of this launch: row-tile major, column tile minor (CTAs that run side by side share the A rows
-// and sweep the expert's B columns, which then sit in L2 for the expert's other row tiles).
-__device__ __forceinline__ bool decode_tile(const GGParams& P, const SmemGG& sm, int idx, int n_tiles, Tile& t) {
+// idx-th work item of this launch: row-tile major, column tile minor (pairs that run side by side share the A rows
+// and sweep the expert's B columns, which then sit in L2 for the expert's other row tiles).  With `tail_split`,
+// the tiles left over after the last full round (every pair one tile) are handed out as half-width items when
+// that lets the leftover round finish in half the time.
+__device__ __forceinline__ bool decode_tile(const GGParams& P, const SmemGG& sm, int idx, int n_tiles, int n_pairs, Tile& t) {
   const int per_row = n_tiles * P.ksplit;
+  int half = -1;
+  if (P.tail_split) {
+    const int total = sm.tile_prefix[P.E] * per_row;
+    const int full = total / n_pairs * n_pairs;
+    if (2 * (total - full) <= n_pairs && idx >= full) {
+      half = (idx - full) & 1;
+      idx = full + ((idx - full) >> 1);
+    }
+  }
   const int mt = idx / per_row, rem = idx - mt * per_row;
   const int nt = rem / P.ksplit;
   t.ks = rem - nt * P.ksplit;
   if (mt >= sm.tile_prefix[P.E]) return false;
   int e = 0;
   while (sm.tile_prefix[e + 1] <= mt) ++e;
-  const int tile_rows = P.tile_rows;
   t.e = e;
-  t.m0 = P.offsets[e] + (mt - sm.tile_prefix[e]) * tile_rows;
+  t.m0 = P.offsets[e] + (mt - sm.tile_prefix[e]) * kPairRows;
   t.m_end = P.offsets[e + 1];
-  t.halves = (!P.dual_a && tile_rows > kBM && t.m_end - t.m0 > kBM) ? 2 : 1;
   t.n0 = nt * P.bn;
+  t.bn = P.bn;
+  if (half >= 0) t.bn = P.bn / 2, t.n0 += half * t.bn;
   return true;
 }
 
 __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
 
-// Persistent: CTA c takes tiles c, c + gridDim.x, ...; the TMA producer runs ahead into the next tile while
-// the epilogue of the current one drains TMEM.
 __global__ void __launch_bounds__(kThreadsGG, 1)
     grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                         const __grid_constant__ CUtensorMap map_b, const GGParams P) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  // stage layout: [A 16 KB][A' 16 KB][B 32 KB], all 1024-byte aligned (swizzle atoms).  A' is the second
-  // 128-row half of the tile, or the second operand (dual_a, 128-row tiles)
-  const uint32_t a_bytes = kBM * kBK * 2, b_bytes = 256 * kBK * 2;
-  // (tiles of one 128-row half with a single A operand leave A' out: stages of 48 KB, one more of them)
-  const uint32_t n_a = P.single_a ? 1u : 2u;
-  const uint32_t stage_bytes = n_a * a_bytes + b_bytes;
+  // stage layout: [A 16 KB][A' 16 KB, B_DUAL only][B <= 16 KB], all 1024-byte aligned (swizzle atoms); identical
+  // in both CTAs, because the MMA addresses the pair's operands by one shared-memory offset
+  const uint32_t a_bytes = kBM * kBK * 2;
+  const uint32_t n_a = P.bmode == B_DUAL ? 2u : 1u;
+  const uint32_t b_rows = (P.bmode == B_PAIR || P.bmode == B_DUAL) ? (uint32_t)P.bn : (uint32_t)P.bn / 2u;  // per CTA
+  const uint32_t b_bytes = b_rows * kBK * 2;
+  const uint32_t stage_bytes = n_a * a_bytes + 128u * kBK * 2u;
   unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   SmemGG& sm = *reinterpret_cast<SmemGG*>(stages + (size_t)P.n_stages * stage_bytes);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NS = P.n_stages;
   const int num_kb = (P.K + kBK - 1) / kBK;
   const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   pdl_launch_dependents();
   if (tid == 0) {
@@ -195,284 +243,265 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       mbar_init(&sm.full[i], 1);
       mbar_init(&sm.empty[i], 1);
     }
-    for (int i = 0; i < kTileQueue; ++i) {
-      mbar_init(&sm.tq_full[i], 1);
-      mbar_init(&sm.tq_empty[i], 1 + kEpiWarps);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sm.accum_full[b], 1);
+      mbar_init(&sm.accum_empty[b], 2 * kEpiWarps);
     }
-    mbar_init(&sm.accum_full, 1);
-    mbar_init(&sm.accum_empty, kEpiWarps);
     sm.abort = 0;
     fence_mbar_init();
     fence_proxy_async_smem();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
+  if (warp == 1) {  // one warp of each CTA of the pair
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                  "n"(kTmemCols)
                  : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   // everything above touches only this CTA's shared memory and TMEM; the expert offsets and the operands may
   // come from the kernel before
   pdl_wait();
   if (tid == 0) {
-    if (blockIdx.x == 0) P.st->tile_ctr[P.ctr_idx ^ 1] = 0u;  // for the next GEMM of the chain (it starts after this one ends)
     int run = 0;
     for (int i = 0; i < P.E; ++i) {
       sm.tile_prefix[i] = run;
       const int rows = P.offsets[i + 1] - P.offsets[i];
-      run += rows > 0 ? (rows + P.tile_rows - 1) / P.tile_rows : 0;
+      run += rows > 0 ? (rows + kPairRows - 1) / kPairRows : 0;
     }
     sm.tile_prefix[P.E] = run;
   }
   tc_fence_before();
   __syncthreads();
+  __syncwarp();
+  cluster_sync_all();  // the other CTA's barriers are initialised before anything is counted on them
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
   Tile t;
 
   if (warp == 0) {
-    // ================================================================= TMA producer
+    // ================================================================= TMA producer (both CTAs)
     if (lane == 0) {
-      int it = 0;  // k-blocks issued so far, over all tiles
+      int it = 0;              // k-blocks issued so far, over all tiles
+      uint32_t slot = 0, par = 1;  // ring position; parity of the `empty` phase the slot's next fill waits for
       bool ok = true;
-      // Tiles are drawn from a counter in global memory (the CTAs' tiles differ in cost: one or two halves, operands
-      // found in L2 or not) and passed on to the MMA thread and the epilogue warps through a small queue.
-      for (int ti = 0; ok; ++ti) {
-        const int qs = ti % kTileQueue;
-        if (ti >= kTileQueue && !mbar_wait(&sm.tq_empty[qs], ((ti / kTileQueue) - 1) & 1)) {
-          flag_error(P.st, MOE_ERR_TIMEOUT, 0x404u);
-          sm.abort = 1;
-          ok = false;
-          break;
-        }
-        const int idx = (int)atomicAdd(&P.st->tile_ctr[P.ctr_idx], 1u);
-        sm.tq[qs] = idx;
-        mbar_arrive(&sm.tq_full[qs]);
-        if (!decode_tile(P, sm, idx, n_tiles, t)) break;  // past the last tile: the others stop on it too
-        const uint32_t tx = a_bytes * (P.dual_a ? 2 : t.halves) +
-                            (P.pair ? 2u * 128u * kBK * 2u : (uint32_t)P.bn * kBK * 2u);
+      const uint32_t full0 = map_to_rank(&sm.full[0], 0u);      // the leader's stage barriers, 8 bytes apart
+      const int half_bn = P.bn / 2;
+      for (int idx = pair; ok && decode_tile(P, sm, idx, n_tiles, n_pairs, t); idx += n_pairs) {
         const int kb0 = t.ks * num_kb / P.ksplit, kb1 = (t.ks + 1) * num_kb / P.ksplit;
+        const int a_row = t.m0 + (int)rank * kBM;
+        // bytes both CTAs bring in per stage (a half-width tile of the last round has half the B bytes)
+        const uint32_t tx_pair = 2u * (n_a * a_bytes + (t.bn == P.bn ? b_bytes : b_bytes / 2u));
+        int k0 = kb0 * kBK;
+        int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % NS;
-          if (it >= NS && !mbar_wait(&sm.empty[s], ((it / NS) - 1) & 1)) {
+          if (it >= NS && !mbar_wait(&sm.empty[slot], par)) {
             flag_error(P.st, MOE_ERR_TIMEOUT, 0x400u);
             sm.abort = 1;
             ok = false;
             break;
           }
-          unsigned char* st_a0 = stages + (size_t)s * stage_bytes;
-          unsigned char* st_a1 = st_a0 + a_bytes;
+          unsigned char* st_a0 = stages + (size_t)slot * stage_bytes;
           unsigned char* st_b = st_a0 + n_a * a_bytes;
-          const int k0 = kb * kBK;
-          const int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
-          mbar_arrive_expect_tx(&sm.full[s], tx);
-          tma_load_2d(st_a0, &map_a0, k0, t.m0, &sm.full[s]);
-          if (P.dual_a)
-            tma_load_2d(st_a1, &map_a1, k0, t.m0, &sm.full[s]);
-          else if (t.halves == 2)
-            tma_load_2d(st_a1, &map_a0, k0, t.m0 + kBM, &sm.full[s]);
-          if (P.b_nmajor) {
-            for (int j = 0; j < P.bn / 64; ++j)
-              tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, t.n0 + 64 * j, P.b_sub, kB, t.e, &sm.full[s]);
-          } else if (P.pair) {
-            tma_load_4d(st_b, &map_b, kB, 0, t.n0, t.e, &sm.full[s]);
-            tma_load_4d(st_b + 128 * kBK * 2, &map_b, kB, 1, t.n0, t.e, &sm.full[s]);
+          const uint32_t bar = full0 + 8u * slot;
+          if (rank == 0) mbar_arrive_expect_tx(&sm.full[slot], tx_pair);
+          tma_load_2d(st_a0, &map_a0, k0, a_row, bar);
+          if (P.bmode == B_PAIR) {
+            tma_load_4d(st_b, &map_b, kB, (int)rank, t.n0, t.e, bar);
+          } else if (P.bmode == B_DUAL) {
+            const int nr = t.n0 + (int)rank * half_bn;
+            tma_load_2d(st_a0 + a_bytes, &map_a1, k0, a_row, bar);
+            tma_load_4d(st_b, &map_b, kB, 0, nr, t.e, bar);
+            tma_load_4d(st_b + (size_t)half_bn * kBK * 2, &map_b, kB, 1, nr, t.e, bar);
+          } else if (P.bmode == B_SINGLE) {
+            tma_load_4d(st_b, &map_b, kB, P.b_sub, t.n0 + (int)rank * half_bn, t.e, bar);
           } else {
-            tma_load_4d(st_b, &map_b, kB, P.b_sub, t.n0, t.e, &sm.full[s]);
+            const int nc = t.n0 + (int)rank * (t.bn / 2);
+            for (int j = 0; j < t.bn / 128; ++j)
+              tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, nc + 64 * j, P.b_sub, kB, t.e, bar);
           }
+          k0 += kBK, kB += kBK;
+          if (P.k_wrap > 0 && kB >= P.k_wrap) kB -= P.k_wrap;
+          if (++slot == (uint32_t)NS) slot = 0, par ^= 1u;
         }
       }
-      if (!ok) {  // copies in flight must land before the CTA goes away
+      if (!ok && rank == 0) {  // copies in flight (both CTAs' complete on these barriers) must land before the pair goes away
         for (int j = max(0, it - NS); j < it; ++j) (void)mbar_wait(&sm.full[j % NS], (j / NS) & 1);
       }
     }
   } else if (warp == 1) {
-    // ================================================================= MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc_pairhalf = instr_desc(128, false);
-      const uint32_t idesc_single = instr_desc(P.pair ? 256 : P.bn, P.b_nmajor != 0);
-      int it = 0, tile_i = 0;
+    // ================================================================= MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      // One thread feeds the tensor cores of both SMs, so its instruction stream is kept short: the ring position
+      // is a counter, not a division, and the operand descriptors are a constant high word plus a low word that
+      // steps through the stage (K-major operands: 32 bytes per 16 k-values; N-major: 16 k-rows of 128 bytes).
+      const int n_mma = P.bmode == B_PAIR ? 2 * P.bn : P.bn;
+      const uint32_t idesc_full = instr_desc(n_mma, P.bmode == B_NMAJOR), idesc_half = instr_desc(n_mma / 2, P.bmode == B_NMAJOR);
+      const uint64_t hi_k = smem_desc(0, 16, 1024) & 0xffffffff00000000ull;
+      const uint64_t hi_b = (P.bmode == B_NMAJOR ? smem_desc(0, 64 * kBK * 2, 1024) : smem_desc(0, 16, 1024)) & 0xffffffff00000000ull;
+      const uint32_t lo_b_lbo = (P.bmode == B_NMAJOR ? (uint32_t)(64 * kBK * 2 >> 4) : 1u) << 16;
+      const uint32_t b_step = P.bmode == B_NMAJOR ? (2048u >> 4) : (32u >> 4);
+      const uint32_t stage0 = smem_u32(stages) >> 4, stage_step = stage_bytes >> 4;
+      const uint32_t b_off = (n_a * a_bytes) >> 4, a1_off = a_bytes >> 4, b1_off = ((uint32_t)(P.bn / 2) * kBK * 2) >> 4;
+      uint32_t slot = 0, par = 0, st_lo = stage0;
+      int tile_i = 0;
       bool ok = true;
-      for (;; ++tile_i) {
-        const int qs = tile_i % kTileQueue;
-        if (!ok) break;
-        if (!mbar_wait(&sm.tq_full[qs], (tile_i / kTileQueue) & 1)) {
-          flag_error(P.st, MOE_ERR_TIMEOUT, 0x405u);
-          sm.abort = 1;
-          break;
-        }
-        const int idx = sm.tq[qs];
-        mbar_arrive(&sm.tq_empty[qs]);
-        if (!decode_tile(P, sm, idx, n_tiles, t)) break;
-        if (tile_i > 0) {  // the previous tile's accumulators must have left TMEM
-          if (!mbar_wait(&sm.accum_empty, (tile_i - 1) & 1)) {
+      for (int idx = pair; ok && decode_tile(P, sm, idx, n_tiles, n_pairs, t); idx += n_pairs, ++tile_i) {
+        const int buf = tile_i & 1;
+        if (tile_i >= 2) {  // the accumulators two tiles back must have left this buffer, in both CTAs
+          if (!mbar_wait(&sm.accum_empty[buf], ((tile_i >> 1) - 1) & 1)) {
             flag_error(P.st, MOE_ERR_TIMEOUT, 0x403u);
             sm.abort = 1;
-            ok = false;
             break;
           }
           tc_fence_after();
         }
+        const uint32_t d_tmem = tmem + (uint32_t)(buf * kAccCols);
         const int kb0 = t.ks * num_kb / P.ksplit, kb1 = (t.ks + 1) * num_kb / P.ksplit;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % NS;
-          if (!mbar_wait(&sm.full[s], (it / NS) & 1)) {
+        const uint32_t idesc = t.bn == P.bn ? idesc_full : idesc_half;
+        uint32_t acc = 0;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(&sm.full[slot], par)) {
             flag_error(P.st, MOE_ERR_TIMEOUT, 0x401u);
             sm.abort = 1;
             ok = false;
             break;
           }
           tc_fence_after();
-          const uint32_t a0 = smem_u32(stages + (size_t)s * stage_bytes);
-          const uint32_t a1 = a0 + a_bytes;
-          const uint32_t b = a0 + n_a * a_bytes;
+          const uint64_t da = hi_k | (uint64_t)(st_lo | (1u << 16));
+          const uint64_t db = hi_b | (uint64_t)((st_lo + b_off) | lo_b_lbo);
+          if (P.bmode == B_DUAL) {
+            const uint64_t da1 = da + a1_off, db1 = db + b1_off;
 #pragma unroll
-          for (int kk = 0; kk < kBK / 16; ++kk) {
-            const bool acc = (kb > kb0) || (kk > 0);
-            const uint64_t da0 = smem_desc(a0 + kk * 32, 16, 1024);
-            if (P.b_nmajor) {
-              const uint64_t db = smem_desc(b + kk * 2048, 64 * kBK * 2, 1024);
-              tc_mma_bf16(tmem, da0, db, idesc_single, acc);
-              if (t.halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
-            } else if (P.dual_a) {
-              const uint64_t da1 = smem_desc(a1 + kk * 32, 16, 1024);
-              const uint64_t db0 = smem_desc(b + kk * 32, 16, 1024);
-              const uint64_t db1 = smem_desc(b + 128 * kBK * 2 + kk * 32, 16, 1024);
-              tc_mma_bf16(tmem, da0, db0, idesc_pairhalf, acc);
-              tc_mma_bf16(tmem + 128, da1, db1, idesc_pairhalf, acc);
-            } else {
-              const uint64_t db = smem_desc(b + kk * 32, 16, 1024);
-              tc_mma_bf16(tmem, da0, db, idesc_single, acc);
-              if (t.halves == 2) tc_mma_bf16(tmem + 256, smem_desc(a1 + kk * 32, 16, 1024), db, idesc_single, acc);
+            for (uint32_t kk = 0; kk < kBK / 16; ++kk) {
+              tc_mma_bf16(d_tmem, da + 2u * kk, db + 2u * kk, idesc, acc | kk);
+              tc_mma_bf16(d_tmem + (uint32_t)P.bn, da1 + 2u * kk, db1 + 2u * kk, idesc, acc | kk);
             }
+          } else {
+#pragma unroll
+            for (uint32_t kk = 0; kk < kBK / 16; ++kk) tc_mma_bf16(d_tmem, da + 2u * kk, db + b_step * kk, idesc, acc | kk);
           }
-          tc_commit(&sm.empty[s]);  // arrives when the MMAs above have finished reading this stage
+          acc = 1;
+          tc_commit_pair(&sm.empty[slot]);  // both CTAs' producers may refill the stage once these MMAs have read it
+          st_lo += stage_step;
+          if (++slot == (uint32_t)NS) slot = 0, par ^= 1u, st_lo = stage0;
         }
-        if (ok) tc_commit(&sm.accum_full);
+        if (ok) tc_commit_pair(&sm.accum_full[buf]);
       }
     }
   } else {
-    // ================================================================= epilogue (warps 2..9)
+    // ================================================================= epilogue (warps 2..9, both CTAs)
     const int q = warp & 3;  // TMEM lanes 32q .. 32q+31 are the only ones this warp may read
     const int cpar = (warp - 2) >> 2;  // which of the two warps of this quarter: it takes every other 32-column chunk
+    const uint32_t acce_bar[2] = {map_to_rank(&sm.accum_empty[0], 0u), map_to_rank(&sm.accum_empty[1], 0u)};
     int tile_i = 0;
-    for (;; ++tile_i) {
-      const int qs = tile_i % kTileQueue;
-      if (!mbar_wait(&sm.tq_full[qs], (tile_i / kTileQueue) & 1)) {
-        if (lane == 0) flag_error(P.st, MOE_ERR_TIMEOUT, 0x406u);
-        break;
-      }
-      const int idx = sm.tq[qs];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.tq_empty[qs]);
-      if (!decode_tile(P, sm, idx, n_tiles, t)) break;
-      if (!mbar_wait(&sm.accum_full, tile_i & 1)) {
+    for (int idx = pair; decode_tile(P, sm, idx, n_tiles, n_pairs, t); idx += n_pairs, ++tile_i) {
+      const int buf = tile_i & 1;
+      if (!mbar_wait(&sm.accum_full[buf], (tile_i >> 1) & 1)) {
         if (lane == 0) flag_error(P.st, MOE_ERR_TIMEOUT, 0x402u);
         break;
       }
       tc_fence_after();
-      const int ncols = min(P.bn, P.n_total - t.n0);  // valid columns of this tile (multiple of 8)
-      for (int hf = 0; hf < t.halves; ++hf) {
-        const int row = t.m0 + hf * kBM + 32 * q + lane;
-        const bool row_ok = row < t.m_end;
-        const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(hf * 256);
-        if (P.epi == EPI_SWIGLU || P.epi == EPI_BF16_PAIR) {
-          __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + t.n0;
-          for (int c = 32 * cpar; c < P.bn; c += 64) {
-            uint32_t g[32], u[32];
-            tc_ld32(tbase + c, g);
-            tc_ld32(tbase + 128 + c, u);
-            tc_wait_ld();
-            if (!row_ok) continue;
-            if (P.epi == EPI_SWIGLU) {
+      const int ncols = min(t.bn, P.n_store - t.n0);  // columns of this tile to store (multiple of 8)
+      const int row = t.m0 + (int)rank * kBM + 32 * q + lane;
+      const bool row_ok = row < t.m_end;
+      const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kAccCols);
+      if (P.epi == EPI_SWIGLU || P.epi == EPI_BF16_PAIR) {
+        __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + t.n0;
+        for (int c = 32 * cpar; c < P.bn; c += 64) {
+          uint32_t g[32], u[32];
+          tc_ld32(tbase + c, g);
+          tc_ld32(tbase + P.bn + c, u);
+          tc_wait_ld();
+          if (!row_ok) continue;
+          if (P.epi == EPI_SWIGLU) {
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                if (c + 8 * v < ncols) {
-                  uint32_t o[4];
+            for (int v = 0; v < 4; ++v) {
+              if (c + 8 * v < ncols) {
+                uint32_t o[4];
 #pragma unroll
-                  for (int j = 0; j < 4; ++j)
-                    o[j] = pack_bf16x2(
-                        silu_mul(__uint_as_float(g[8 * v + 2 * j]), __uint_as_float(u[8 * v + 2 * j])),
-                        silu_mul(__uint_as_float(g[8 * v + 2 * j + 1]), __uint_as_float(u[8 * v + 2 * j + 1])));
-                  *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
-                }
+                for (int j = 0; j < 4; ++j)
+                  o[j] = pack_bf16x2(silu_mul(__uint_as_float(g[8 * v + 2 * j]), __uint_as_float(u[8 * v + 2 * j])),
+                                     silu_mul(__uint_as_float(g[8 * v + 2 * j + 1]), __uint_as_float(u[8 * v + 2 * j + 1])));
+                *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
               }
-            } else {
+            }
+          } else {
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                if (c + 8 * v < ncols) {
-                  uint32_t o[4], p[4];
+            for (int v = 0; v < 4; ++v) {
+              if (c + 8 * v < ncols) {
+                uint32_t o[4], p[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  o[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]), __uint_as_float(g[8 * v + 2 * j + 1]));
+                  p[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]), __uint_as_float(u[8 * v + 2 * j + 1]));
+                }
+                *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(out + P.out_off2 + c + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
+                if (P.split) {
+                  uint32_t ol[4], pl[4];
 #pragma unroll
                   for (int j = 0; j < 4; ++j) {
-                    o[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]), __uint_as_float(g[8 * v + 2 * j + 1]));
-                    p[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]), __uint_as_float(u[8 * v + 2 * j + 1]));
+                    ol[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
+                                        __uint_as_float(g[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
+                    pl[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]) - __uint_as_float(p[j] << 16),
+                                        __uint_as_float(u[8 * v + 2 * j + 1]) - __uint_as_float(p[j] & 0xffff0000u));
                   }
-                  *reinterpret_cast<uint4*>(out + c + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
-                  *reinterpret_cast<uint4*>(out + P.out_off2 + c + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
-                  if (P.split) {
-                    uint32_t ol[4], pl[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                      ol[j] = pack_bf16x2(__uint_as_float(g[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
-                                          __uint_as_float(g[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
-                      pl[j] = pack_bf16x2(__uint_as_float(u[8 * v + 2 * j]) - __uint_as_float(p[j] << 16),
-                                          __uint_as_float(u[8 * v + 2 * j + 1]) - __uint_as_float(p[j] & 0xffff0000u));
-                    }
-                    *reinterpret_cast<uint4*>(out + P.out_off_lo + c + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-                    *reinterpret_cast<uint4*>(out + P.out_off2 + P.out_off_lo + c + 8 * v) =
-                        make_uint4(pl[0], pl[1], pl[2], pl[3]);
-                  }
+                  *reinterpret_cast<uint4*>(out + P.out_off_lo + c + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                  *reinterpret_cast<uint4*>(out + P.out_off2 + P.out_off_lo + c + 8 * v) =
+                      make_uint4(pl[0], pl[1], pl[2], pl[3]);
                 }
               }
             }
           }
-        } else {
-          for (int c = 32 * cpar; c < P.bn; c += 64) {
-            uint32_t a[32];
-            tc_ld32(tbase + c, a);
-            tc_wait_ld();
-            if (!row_ok) continue;
-            if (P.epi == EPI_F32) {
-              float* out = (float*)P.out + (size_t)t.ks * P.plane_elems + (size_t)row * P.ld_out + t.n0 + c;
+        }
+      } else {
+        for (int c = 32 * cpar; c < t.bn; c += 64) {
+          uint32_t a[32];
+          tc_ld32(tbase + c, a);
+          tc_wait_ld();
+          if (!row_ok) continue;
+          if (P.epi == EPI_F32) {
+            float* out = (float*)P.out + (size_t)t.ks * P.plane_elems + (size_t)row * P.ld_out + t.n0 + c;
 #pragma unroll
-              for (int v = 0; v < 8; ++v)
-                if (c + 4 * v < ncols)
-                  *reinterpret_cast<uint4*>(out + 4 * v) = make_uint4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
-            } else {
-              __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + t.n0 + c;
+            for (int v = 0; v < 8; ++v)
+              if (c + 4 * v < ncols)
+                *reinterpret_cast<uint4*>(out + 4 * v) = make_uint4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
+          } else {
+            __nv_bfloat16* out = (__nv_bfloat16*)P.out + (size_t)row * P.ld_out + t.n0 + c;
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                if (c + 8 * v < ncols) {
-                  uint32_t o[4];
+            for (int v = 0; v < 4; ++v) {
+              if (c + 8 * v < ncols) {
+                uint32_t o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  o[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]), __uint_as_float(a[8 * v + 2 * j + 1]));
+                *reinterpret_cast<uint4*>(out + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
+                if (P.split) {
+                  uint32_t ol[4];
 #pragma unroll
                   for (int j = 0; j < 4; ++j)
-                    o[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]), __uint_as_float(a[8 * v + 2 * j + 1]));
-                  *reinterpret_cast<uint4*>(out + 8 * v) = make_uint4(o[0], o[1], o[2], o[3]);
-                  if (P.split) {
-                    uint32_t ol[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                      ol[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
-                                          __uint_as_float(a[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
-                    *reinterpret_cast<uint4*>(out + P.out_off_lo + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-                  }
+                    ol[j] = pack_bf16x2(__uint_as_float(a[8 * v + 2 * j]) - __uint_as_float(o[j] << 16),
+                                        __uint_as_float(a[8 * v + 2 * j + 1]) - __uint_as_float(o[j] & 0xffff0000u));
+                  *reinterpret_cast<uint4*>(out + P.out_off_lo + 8 * v) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
                 }
               }
             }
           }
         }
       }
-      // the accumulators are in registers / memory now: hand TMEM back to the MMA warp
+      // the accumulators are in registers / memory now: hand the buffer back to the leader's MMA thread
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.accum_empty);
+      if (lane == 0) mbar_arrive_cluster(acce_bar[buf]);
     }
   }
-  // ---- teardown: every role gets here in bounded time
+  // ---- teardown: every role gets here in bounded time; neither CTA leaves while the other may still count on
+  // its barriers or read its operands
   tc_fence_before();
   __syncthreads();
+  __syncwarp();
+  cluster_sync_all();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kTmemCols) : "memory");
   }
 }
 
@@ -525,36 +554,58 @@ int make_map_b(CUtensorMap* m, const void* base, long long inner, int nsub, long
   return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
 }
 
+// Pairs of CTAs the device can hold at once (one CTA per SM; a pair sits on two SMs of one cluster).
+void pair_launch_config(cudaLaunchConfig_t& lc, cudaLaunchAttribute* attr, int ctas, size_t smem, cudaStream_t s) {
+  lc = cudaLaunchConfig_t{};
+  lc.gridDim = dim3(ctas), lc.blockDim = dim3(kThreadsGG), lc.dynamicSmemBytes = smem, lc.stream = s;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr, lc.numAttrs = 2;
+}
+
+// Pairs of CTAs the device can hold at once (one CTA per SM; a pair sits on two SMs of one cluster).
+int max_pairs(moe_ctx* ctx, size_t smem) {
+  cudaLaunchConfig_t lc;
+  cudaLaunchAttribute attr[2];
+  pair_launch_config(lc, attr, ctx->sm_count & ~1, smem, nullptr);
+  lc.numAttrs = 1;  // the cluster shape alone decides the occupancy
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, grouped_gemm_kernel, &lc) != cudaSuccess || n < 1) {
+    (void)cudaGetLastError();
+    n = ctx->sm_count / 2;
+  }
+  return std::max(1, std::min(n, ctx->sm_count / 2));
+}
+
 int launch_gg(moe_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b, GGParams P,
               int n_slots, cudaStream_t s) {
   const moe_config& c = ctx->cfg;
   P.E = c.n_experts;
   P.st = ctx->d_state;
-  const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
-  // 256-row tiles read every B slice once for up to 256 rows of an expert (half the operand traffic per flop,
-  // and an expert with 129..256 rows is one tile instead of two); problems whose 256-row tiles would leave SMs
-  // without work keep 128-row tiles.  A cut contraction (ksplit) multiplies the work items.
-  P.tile_rows = kBM;
+  if (P.n_store < P.n_total) P.n_store = P.n_total;
   if (P.ksplit < 1) P.ksplit = 1;
-  const long long m256 = std::max<long long>((n_slots + kTileRows - 1) / kTileRows, std::min(c.n_experts, n_slots));
-  if (!P.dual_a && (m256 * n_tiles >= ctx->sm_count || P.ksplit > 1)) P.tile_rows = kTileRows;
-  P.single_a = (P.tile_rows == kBM && !P.dual_a) ? 1 : 0;
-  P.n_stages = P.single_a ? 4 : 3;
-  const size_t stage_bytes = (size_t)kBM * kBK * 2 * (P.single_a ? 1 : 2) + 256 * kBK * 2;
+  const int n_tiles = (P.n_total + P.bn - 1) / P.bn;
+  const size_t stage_bytes = (size_t)kBM * kBK * 2 * (P.bmode == B_DUAL ? 2 : 1) + 128 * kBK * 2;
+  P.n_stages = P.bmode == B_DUAL ? 4 : kMaxStagesGG;
   const size_t smem = P.n_stages * stage_bytes + sizeof(SmemGG) + 1024 + 128;
   if ((long long)smem > ctx->max_smem_optin) return MOE_ERR_UNSUPPORTED;
-  const long long m_tiles = (n_slots + P.tile_rows - 1) / P.tile_rows + c.n_experts;  // upper bound
-  const int grid = (int)std::min<long long>(m_tiles * n_tiles * P.ksplit, ctx->sm_count);
   MOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  MOE_CUDA_TRY(launch_pdl(grouped_gemm_kernel, dim3(grid), dim3(kThreadsGG), smem, s, a0, a1, b, P));
-  MOE_CUDA_TRY(cudaGetLastError());
+  const long long m_tiles = (n_slots + kPairRows - 1) / kPairRows + c.n_experts;  // upper bound
+  const int pairs = (int)std::min<long long>(m_tiles * n_tiles * P.ksplit, max_pairs(ctx, smem));
+  cudaLaunchConfig_t lc;
+  cudaLaunchAttribute attr[2];
+  pair_launch_config(lc, attr, 2 * pairs, smem, s);
+  MOE_CUDA_TRY(cudaLaunchKernelEx(&lc, grouped_gemm_kernel, a0, a1, b, P));
   ctx->launches++;
   return MOE_OK;
 }
 
-int pick_bn(int n_total, int cap) {
+// Output columns per tile: the largest of 64, 128, ... `cap` that is not mostly padding.
+int pick_bn(int n_total, int cap, int floor_bn = 64) {
   int bn = cap;
-  while (bn > 64 && bn / 2 >= n_total) bn /= 2;
+  while (bn > floor_bn && bn / 2 >= n_total) bn /= 2;
   return bn;
 }
 
@@ -576,70 +627,69 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
   GGParams P{};
   P.offsets = offsets;
   if (r == 0) {
-    // (1) hidden = silu(X Wg) * (X Wu)
+    // (1) hidden = silu(X Wg) * (X Wu): the tile's 128 gate rows come in through one CTA, its 128 up rows through the other
     if ((rc = make_map_a(&ma, xperm, n_slots, d, d)) != MOE_OK) return rc;
     if ((rc = make_map_b(&mb, w->gud, d, 3, f, E, kBK, 128)) != MOE_OK) return rc;
-    P.K = d, P.n_total = f, P.bn = 128, P.pair = 1, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_SWIGLU;
+    P.K = d, P.n_total = f, P.bn = 128, P.bmode = B_PAIR, P.b_sub = 0, P.epi = EPI_SWIGLU;
     P.out = hidden, P.ld_out = f, P.out_off2 = 0;
-    P.ctr_idx = 0;
     if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
     // (2) out_slots = hidden Wd   (B = down rows of gud: [k = hidden unit][n = model column], n contiguous)
     if ((rc = make_map_a(&ma, hidden, n_slots, f, f)) != MOE_OK) return rc;
     if ((rc = make_map_b(&mb, w->gud, d, 3, f, E, 64, kBK)) != MOE_OK) return rc;
-    P.K = f, P.n_total = d, P.bn = pick_bn(d, 256), P.pair = 0, P.dual_a = 0, P.b_nmajor = 1, P.b_sub = 2;
+    P.K = f, P.n_total = d, P.bn = pick_bn(d, 256, 128), P.bmode = B_NMAJOR, P.b_sub = 2;
     P.epi = EPI_F32, P.out = out_slots, P.ld_out = d, P.out_off2 = 0;
+    P.tail_split = P.bn == 256 ? 1 : 0;
     if (out_planes && n_slots <= kKSplitMaxSlots) {
       // short prefill: too few tiles for the SMs, and every tile streams a long run of weights.  The caller
-      // sums planes: cut the contraction so that every SM streams a part, each part into its own plane.
-      const int m_est = std::max((n_slots + kBM - 1) / kBM, std::min(E, n_slots));
+      // sums planes: cut the contraction so that every pair streams a part, each part into its own plane.
+      const int m_est = std::max((n_slots + kPairRows - 1) / kPairRows, std::min(E, n_slots));
       const long long tiles = (long long)m_est * ((d + P.bn - 1) / P.bn);
-      int ks = (int)(ctx->sm_count / std::max<long long>(tiles, 1));
+      int ks = (int)((ctx->sm_count / 2) / std::max<long long>(tiles, 1));
       ks = std::min(std::min(ks, kKSplitMax), (f + kBK - 1) / kBK);
       if (ks > 1) {
+        P.tail_split = 0;
         P.ksplit = ks, P.plane_elems = (long long)n_slots * d;
         *out_planes = ks;
       }
     }
-    P.ctr_idx = 1;
     return launch_gg(ctx, ma, ma, mb, P, n_slots, s);
   }
   // The rank-r intermediates t and v are kept as hi + lo pairs of bf16 (value = hi + lo): the GEMMs that
-  // consume them run over K = 2r with the weight slices repeated, so the intermediates carry ~16 mantissa
+  // consume them run over K = 2 * rp with the weight slices repeated, so the intermediates carry ~16 mantissa
   // bits and the chain's only bf16 roundings are those of the dense path (hidden activations, output).
-  const bool split = (r % kBK) == 0;
-  const int tw = split ? 2 * r : r;  // stored width of one intermediate
+  // rp = r rounded up to the K step: the columns [r, rp) of an intermediate are stored as zeros and meet
+  // weight rows past the end of the matrix (zero-filled by the loads), so any rank that is a multiple of 8 works.
+  const int rp = (r + kBK - 1) / kBK * kBK;
+  const int tw = 2 * rp;  // stored width of one intermediate: hi | lo
   void* mid_a = ws + L.mid_a;  // [n_slots][2*tw]: t_g (hi | lo) | t_u (hi | lo)
   void* mid_b = ws + L.mid_b;  // [n_slots][tw]:   v (hi | lo)
   // (1) T = X [gL | uL]
   if ((rc = make_map_a(&ma, xperm, n_slots, d, d)) != MOE_OK) return rc;
-  if ((rc = make_map_b(&mb, w->wd_a, d, 2, r, E, kBK, 128)) != MOE_OK) return rc;
-  P.K = d, P.n_total = r, P.bn = 128, P.pair = 1, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_BF16_PAIR;
-  P.k_wrap = 0, P.split = split, P.out = mid_a, P.ld_out = 2 * tw, P.out_off2 = tw, P.out_off_lo = r;
-  P.ctr_idx = 0;
+  P.bn = pick_bn(r, 128);
+  if ((rc = make_map_b(&mb, w->wd_a, d, 2, r, E, kBK, P.bn)) != MOE_OK) return rc;
+  P.K = d, P.n_total = r, P.bmode = B_PAIR, P.b_sub = 0, P.epi = EPI_BF16_PAIR;
+  P.k_wrap = 0, P.split = 1, P.out = mid_a, P.ld_out = 2 * tw, P.out_off2 = tw, P.out_off_lo = rp, P.n_store = rp;
   if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
-  // (2) hidden = silu(Tg gR) * (Tu uR)
+  // (2) hidden = silu(Tg gR) * (Tu uR): two A operands, each CTA brings half of the gate and half of the up rows
   if ((rc = make_map_a(&ma, mid_a, n_slots, tw, 2 * tw)) != MOE_OK) return rc;
   if ((rc = make_map_a(&ma1, (const __nv_bfloat16*)mid_a + tw, n_slots, tw, 2 * tw)) != MOE_OK) return rc;
-  if ((rc = make_map_b(&mb, w->wd_b, r, 2, f, E, kBK, 128)) != MOE_OK) return rc;
-  P.K = tw, P.n_total = f, P.bn = 128, P.pair = 1, P.dual_a = 1, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_SWIGLU;
-  P.k_wrap = split ? r : 0, P.split = 0, P.out = hidden, P.ld_out = f, P.out_off2 = 0, P.out_off_lo = 0;
-  P.ctr_idx = 1;
+  if ((rc = make_map_b(&mb, w->wd_b, r, 2, f, E, kBK, 64)) != MOE_OK) return rc;
+  P.K = tw, P.n_total = f, P.bn = 128, P.bmode = B_DUAL, P.b_sub = 0, P.epi = EPI_SWIGLU;
+  P.k_wrap = rp, P.split = 0, P.out = hidden, P.ld_out = f, P.out_off2 = 0, P.out_off_lo = 0, P.n_store = 0;
   if ((rc = launch_gg(ctx, ma, ma1, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (3) V = hidden dL
   if ((rc = make_map_a(&ma, hidden, n_slots, f, f)) != MOE_OK) return rc;
   P.bn = pick_bn(r, 256);
-  if ((rc = make_map_b(&mb, w->wd_c, f, 1, r, E, kBK, P.bn)) != MOE_OK) return rc;
-  P.K = f, P.n_total = r, P.pair = 0, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_BF16;
-  P.k_wrap = 0, P.split = split, P.out = mid_b, P.ld_out = tw, P.out_off2 = 0, P.out_off_lo = r;
-  P.ctr_idx = 0;
+  if ((rc = make_map_b(&mb, w->wd_c, f, 1, r, E, kBK, P.bn / 2)) != MOE_OK) return rc;
+  P.K = f, P.n_total = r, P.bmode = B_SINGLE, P.b_sub = 0, P.epi = EPI_BF16;
+  P.k_wrap = 0, P.split = 1, P.out = mid_b, P.ld_out = tw, P.out_off2 = 0, P.out_off_lo = rp, P.n_store = rp;
   if ((rc = launch_gg(ctx, ma, ma, mb, P, n_slots, s)) != MOE_OK) return rc;
   // (4) out_slots = V dR
   if ((rc = make_map_a(&ma, mid_b, n_slots, tw, tw)) != MOE_OK) return rc;
   P.bn = pick_bn(d, 256);
-  if ((rc = make_map_b(&mb, w->wd_d, r, 1, d, E, kBK, P.bn)) != MOE_OK) return rc;
-  P.K = tw, P.n_total = d, P.pair = 0, P.dual_a = 0, P.b_nmajor = 0, P.b_sub = 0, P.epi = EPI_F32;
-  P.k_wrap = split ? r : 0, P.split = 0, P.out = out_slots, P.ld_out = d, P.out_off2 = 0, P.out_off_lo = 0;
-  P.ctr_idx = 1;
+  if ((rc = make_map_b(&mb, w->wd_d, r, 1, d, E, kBK, P.bn / 2)) != MOE_OK) return rc;
+  P.K = tw, P.n_total = d, P.bmode = B_SINGLE, P.b_sub = 0, P.epi = EPI_F32;
+  P.k_wrap = rp, P.split = 0, P.out = out_slots, P.ld_out = d, P.out_off2 = 0, P.out_off_lo = 0, P.n_store = 0;
   return launch_gg(ctx, ma, ma, mb, P, n_slots, s);
 }
 

@@ -51,6 +51,7 @@ def test_stacked_decode_with_offload_matches_checker(slots):
             if not tie:
                 assert sel[l] == ora["topk_idx"][0].tolist(), (step, l, sel[l], ora["topk_idx"][0])
             else:
+                U.assert_valid_tied_selection(sel[l], ora["logits"][0], sh.top_k, (step, l))
                 ora = O.layer_forward(xin, host[l]["w_router"], host[l]["b_router"], ex, sh.top_k,
                                       forced_topk=np.int32([sel[l]]))
             y_b = torch.from_numpy(ora["y"][0].astype(np.float32)).to(torch.bfloat16).double().numpy()
