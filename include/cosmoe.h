@@ -226,9 +226,19 @@ int moe_stack_decode_step_trace(moe_offload* off, moe_ctx* ctx, const moe_weight
 
 /* ---- routing-trace metrics (Eq. 4-5, Section 2.3 / 3.3) ---------------------------
  * topk_trace dev [B][T][k] int32.  Writes H (Eq. 4, summed over experts) to
- * h_total_out dev [1] uint64; replacements = H / 2 and H_norm = (H/2) / (B k (T-1)). */
+ * h_total_out dev [1] uint64; replacements = H / 2 and H_norm = (H/2) / (B k (T-1)).
+ * A row is read as a set: a repeated id counts once, an id outside [0, n_experts) not at all. */
 int moe_expert_replacements(const int32_t* topk_trace, int32_t B, int32_t T, int32_t k, int32_t n_experts,
                             unsigned long long* h_total_out, void* stream);
+
+/* Expert balance of a routing trace (Section 3.3, "delta between the uniform distribution and the realised
+ * expert balance"; Table 3 and Fig. 6 report it per layer).  topk_trace dev [B][T][k] int32, one row b per
+ * layer.  counts_out dev [B][E] uint64: selections of expert e in row b (integer-exact).  delta_out dev [B+1]
+ * fp64: delta_out[b] = 100 * mean_e |counts[b][e] / sum_e counts[b][e] - 1/E|, delta_out[B] = their mean.
+ * bad_out dev [1] uint64: ids outside [0, E) met (they are not counted).  The paper prints no formula for
+ * this metric: the mean absolute deviation is this library's reading, and no value of the paper pins it.  */
+int moe_delta_uniform(const int32_t* topk_trace, int32_t B, int32_t T, int32_t k, int32_t n_experts,
+                      unsigned long long* counts_out, double* delta_out, unsigned long long* bad_out, void* stream);
 
 #ifdef __cplusplus
 }

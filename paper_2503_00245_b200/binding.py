@@ -68,6 +68,7 @@ _SIGS = {
     "moe_stack_decode_step_trace": (C.c_int, [_P, _P, C.POINTER(moe_weights), _P, C.POINTER(C.c_int32), _P, C.c_size_t,
                                               _P]),
     "moe_expert_replacements": (C.c_int, [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P]),
+    "moe_delta_uniform": (C.c_int, [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P]),
 }
 EXPORTS = tuple(_SIGS)
 
@@ -249,3 +250,8 @@ def moe_stack_decode_step_trace(off: int, ctx: int, routers, h, sel, ws, stream=
 def moe_expert_replacements(topk_trace, B, T, k, n_experts, h_total_out, stream=None):
     _ok(_lib().moe_expert_replacements(_ptr(topk_trace), B, T, k, n_experts, _ptr(h_total_out), _stream(stream)),
         "moe_expert_replacements")
+
+
+def moe_delta_uniform(topk_trace, B, T, k, n_experts, counts_out, delta_out, bad_out, stream=None):
+    _ok(_lib().moe_delta_uniform(_ptr(topk_trace), B, T, k, n_experts, _ptr(counts_out), _ptr(delta_out),
+                                 _ptr(bad_out), _stream(stream)), "moe_delta_uniform")

@@ -16,7 +16,7 @@
 struct moe_offload {
   moe_config cfg;
   int n_layers, slots, E;
-  const void* const* host_experts;
+  std::vector<const void*> host_experts;    // [n_layers][E] pinned master copies (the pointers are copied on creation)
   unsigned char* device_slots;
   size_t slot_bytes;
   cudaStream_t copy_stream;
@@ -52,6 +52,15 @@ __global__ void forced_routing_kernel(const float* __restrict__ probs, int k, in
   }
 }
 
+// A layer's expert -> slot table, passed BY VALUE: every queued update carries its own copy, so a later call
+// for the same layer cannot change what an earlier, still pending update writes.
+struct SlotTable {
+  int32_t slot[MOE_MAX_EXPERTS];
+};
+__global__ void slot_table_kernel(int32_t* __restrict__ table, int E, SlotTable t) {
+  if ((int)threadIdx.x < E) table[threadIdx.x] = t.slot[threadIdx.x];
+}
+
 // u = h / sqrt(mean(h^2)) -> x (bf16 or fp32); one CTA
 __global__ void rms_glue_kernel(const float* __restrict__ h, int d, void* __restrict__ x, int x_is_bf16) {
   __shared__ float s_part[32];
@@ -78,8 +87,9 @@ __global__ void residual_kernel(float* __restrict__ h, const void* __restrict__ 
 }
 
 // Eq. 4: H = sum_b sum_t sum_e |[e in S(b,t+1)] - [e in S(b,t)]| = size of the symmetric difference of
-// consecutive selections, summed.
-__global__ void replacements_kernel(const int32_t* __restrict__ trace, int B, int T, int k,
+// consecutive selections, summed.  A row is read as a SET of experts in [0, E): a repeated id counts once and an
+// id outside the range not at all, exactly as in the 0/1 activity matrix the equation is written on.
+__global__ void replacements_kernel(const int32_t* __restrict__ trace, int B, int T, int k, int E,
                                     unsigned long long* __restrict__ out) {
   unsigned long long local = 0;
   const long long pairs = (long long)B * (T - 1);
@@ -88,13 +98,64 @@ __global__ void replacements_kernel(const int32_t* __restrict__ trace, int B, in
     const long long b = i / (T - 1), t = i % (T - 1);
     const int32_t* s0 = trace + (b * T + t) * k;
     const int32_t* s1 = s0 + k;
-    int common = 0;
-    for (int a = 0; a < k; ++a)
-      for (int c = 0; c < k; ++c) common += (s0[a] == s1[c]);
-    local += (unsigned long long)(2 * (k - common));
+    int n0 = 0, n1 = 0, common = 0;
+    for (int a = 0; a < k; ++a) {
+      const int e0 = s0[a], e1 = s1[a];
+      bool first0 = e0 >= 0 && e0 < E, first1 = e1 >= 0 && e1 < E;
+      for (int c = 0; c < a; ++c) first0 &= (s0[c] != e0), first1 &= (s1[c] != e1);
+      n0 += first0, n1 += first1;
+      if (first0) {
+        bool in1 = false;
+        for (int c = 0; c < k; ++c) in1 |= (s1[c] == e0);
+        common += in1;
+      }
+    }
+    local += (unsigned long long)(n0 + n1 - 2 * common);
   }
   for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
   if ((threadIdx.x & 31) == 0 && local) atomicAdd(out, local);
+}
+
+// Expert balance of a routing trace (Section 3.3): per trace row b (a layer), how often each expert was
+// selected.  One CTA per b; integer counts in shared memory, then to global.  Ids outside [0, E) are counted
+// in bad_out instead.
+__global__ void expert_histogram_kernel(const int32_t* __restrict__ trace, int T, int k, int E,
+                                        unsigned long long* __restrict__ counts, unsigned long long* __restrict__ bad_out) {
+  __shared__ unsigned int s_cnt[MOE_MAX_EXPERTS];
+  __shared__ unsigned int s_bad;
+  const int b = blockIdx.x;
+  if (threadIdx.x < MOE_MAX_EXPERTS) s_cnt[threadIdx.x] = 0u;
+  if (threadIdx.x == 0) s_bad = 0u;
+  __syncthreads();
+  const long long n = (long long)T * k;
+  const int32_t* row = trace + (size_t)b * n;
+  for (long long i = threadIdx.x; i < n; i += blockDim.x) {
+    const int e = row[i];
+    if (e >= 0 && e < E)
+      atomicAdd(&s_cnt[e], 1u);
+    else
+      atomicAdd(&s_bad, 1u);
+  }
+  __syncthreads();
+  if ((int)threadIdx.x < E) counts[(size_t)b * E + threadIdx.x] = s_cnt[threadIdx.x];
+  if (threadIdx.x == 0 && s_bad) atomicAdd(bad_out, (unsigned long long)s_bad);
+}
+// delta[b] = 100 * mean_e | counts[b][e] / sum_e counts[b][e] - 1/E |;  delta[B] = mean over b.  fp64, one thread
+// per b, the mean by thread 0 in b order.
+__global__ void delta_uniform_kernel(const unsigned long long* __restrict__ counts, int B, int E, double* __restrict__ delta) {
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    double tot = 0.0;
+    for (int e = 0; e < E; ++e) tot += (double)counts[(size_t)b * E + e];
+    double acc = 0.0;
+    for (int e = 0; e < E; ++e) acc += fabs((tot > 0.0 ? (double)counts[(size_t)b * E + e] / tot : 0.0) - 1.0 / (double)E);
+    delta[b] = acc / (double)E * 100.0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double m = 0.0;
+    for (int b = 0; b < B; ++b) m += delta[b];
+    delta[B] = m / (double)B;
+  }
 }
 
 }  // namespace
@@ -118,7 +179,7 @@ int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_pe
   if (!o) return MOE_ERR_STATE;
   o->cfg = *cfg;
   o->n_layers = n_layers, o->slots = slots_per_layer, o->E = cfg->n_experts;
-  o->host_experts = host_experts;
+  o->host_experts.assign(host_experts, host_experts + (size_t)n_layers * cfg->n_experts);
   o->device_slots = (unsigned char*)device_slots;
   o->slot_bytes = slot_bytes;
   o->fetches = o->bytes = o->hits = 0;
@@ -240,10 +301,10 @@ static int ensure_impl(moe_offload* o, int32_t layer, const int32_t* sel, int32_
     any = true;
   }
   if (any) {
-    int32_t* ht = o->h_tables + (size_t)layer * o->E;
-    for (int x = 0; x < o->E; ++x) ht[x] = slot_of[x];
-    MOE_CUDA_TRY(cudaMemcpyAsync(o->d_tables + (size_t)layer * o->E, ht, sizeof(int32_t) * o->E, cudaMemcpyHostToDevice,
-                                 o->copy_stream));
+    SlotTable tab{};
+    for (int x = 0; x < o->E; ++x) tab.slot[x] = slot_of[x];
+    slot_table_kernel<<<1, MOE_MAX_EXPERTS, 0, o->copy_stream>>>(o->d_tables + (size_t)layer * o->E, o->E, tab);
+    MOE_CUDA_TRY(cudaGetLastError());
     MOE_CUDA_TRY(cudaEventRecord(o->ev_copy, o->copy_stream));
     MOE_CUDA_TRY(cudaStreamWaitEvent(cs, o->ev_copy, 0));
   }
@@ -370,6 +431,21 @@ int moe_stack_decode_step_trace(moe_offload* o, moe_ctx* ctx, const moe_weights*
   return MOE_OK;
 }
 
+int moe_delta_uniform(const int32_t* trace, int32_t B, int32_t T, int32_t k, int32_t n_experts,
+                      unsigned long long* counts_out, double* delta_out, unsigned long long* bad_out, void* stream) {
+  if (!trace || !counts_out || !delta_out || !bad_out || B <= 0 || T <= 0 || k <= 0 || k > MOE_MAX_TOPK || n_experts <= 0 ||
+      n_experts > MOE_MAX_EXPERTS || B > 1024)
+    return MOE_ERR_INVALID_ARG;
+  if ((long long)T * k >= (1ll << 32)) return MOE_ERR_UNSUPPORTED;  // 32-bit counters per CTA
+  cudaStream_t s = (cudaStream_t)stream;
+  MOE_CUDA_TRY(cudaMemsetAsync(bad_out, 0, sizeof(unsigned long long), s));
+  expert_histogram_kernel<<<B, 256, 0, s>>>(trace, T, k, n_experts, counts_out, bad_out);
+  MOE_CUDA_TRY(cudaGetLastError());
+  delta_uniform_kernel<<<1, 256, 0, s>>>(counts_out, B, n_experts, delta_out);
+  MOE_CUDA_TRY(cudaGetLastError());
+  return MOE_OK;
+}
+
 int moe_expert_replacements(const int32_t* trace, int32_t B, int32_t T, int32_t k, int32_t n_experts,
                             unsigned long long* h_total_out, void* stream) {
   if (!trace || !h_total_out || B <= 0 || T <= 0 || k <= 0 || k > MOE_MAX_TOPK || n_experts <= 0)
@@ -379,7 +455,7 @@ int moe_expert_replacements(const int32_t* trace, int32_t B, int32_t T, int32_t 
   if (T < 2) return MOE_OK;
   const long long pairs = (long long)B * (T - 1);
   const int grid = (int)((pairs + 255) / 256 < 1184 ? (pairs + 255) / 256 : 1184);
-  replacements_kernel<<<grid, 256, 0, s>>>(trace, B, T, k, h_total_out);
+  replacements_kernel<<<grid, 256, 0, s>>>(trace, B, T, k, n_experts, h_total_out);
   MOE_CUDA_TRY(cudaGetLastError());
   return MOE_OK;
 }

@@ -70,7 +70,6 @@ struct GGParams {
   long long ld_out;    // elements
   long long out_off2;  // EPI_BF16_PAIR: column offset of the second half
   long long out_off_lo;  // split: column offset of the remainders
-  int tail_split;         // B_NMAJOR, bn = 256: the tiles of the last, partly filled round are cut into two 128-column halves
   int ksplit;             // the contraction is cut into this many parts, each a work item of its own ...
   long long plane_elems;  // ... writing its partial sums plane_elems further on in `out` (EPI_F32 only)
   int n_stages;
@@ -182,24 +181,13 @@ struct SmemGG {
 };
 
 struct Tile {
-  int e, m0, m_end, n0, ks, bn;
+  int e, m0, m_end, n0, ks;
 };
 
-// idx-th work item of this launch: row-tile major, column tile minor (pairs that run side by side share the A rows
-// and sweep the expert's B columns, which then sit in L2 for the expert's other row tiles).  With `tail_split`,
-// the tiles left over after the last full round (every pair one tile) are handed out as half-width items when
-// that lets the leftover round finish in half the time.
-__device__ __forceinline__ bool decode_tile(const GGParams& P, const SmemGG& sm, int idx, int n_tiles, int n_pairs, Tile& t) {
+// idx-th tile of this launch: row-tile major, column tile minor (pairs that run side by side share the A rows
+// and sweep the expert's B columns, which then sit in L2 for the expert's other row tiles).
+__device__ __forceinline__ bool decode_tile(const GGParams& P, const SmemGG& sm, int idx, int n_tiles, Tile& t) {
   const int per_row = n_tiles * P.ksplit;
-  int half = -1;
-  if (P.tail_split) {
-    const int total = sm.tile_prefix[P.E] * per_row;
-    const int full = total / n_pairs * n_pairs;
-    if (2 * (total - full) <= n_pairs && idx >= full) {
-      half = (idx - full) & 1;
-      idx = full + ((idx - full) >> 1);
-    }
-  }
   const int mt = idx / per_row, rem = idx - mt * per_row;
   const int nt = rem / P.ksplit;
   t.ks = rem - nt * P.ksplit;
@@ -210,8 +198,6 @@ __device__ __forceinline__ bool decode_tile(const GGParams& P, const SmemGG& sm,
   t.m0 = P.offsets[e] + (mt - sm.tile_prefix[e]) * kPairRows;
   t.m_end = P.offsets[e + 1];
   t.n0 = nt * P.bn;
-  t.bn = P.bn;
-  if (half >= 0) t.bn = P.bn / 2, t.n0 += half * t.bn;
   return true;
 }
 
@@ -283,13 +269,12 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       int it = 0;              // k-blocks issued so far, over all tiles
       uint32_t slot = 0, par = 1;  // ring position; parity of the `empty` phase the slot's next fill waits for
       bool ok = true;
+      const uint32_t tx_pair = 2u * (n_a * a_bytes + b_bytes);  // bytes both CTAs bring in per stage
       const uint32_t full0 = map_to_rank(&sm.full[0], 0u);      // the leader's stage barriers, 8 bytes apart
       const int half_bn = P.bn / 2;
-      for (int idx = pair; ok && decode_tile(P, sm, idx, n_tiles, n_pairs, t); idx += n_pairs) {
+      for (int idx = pair; ok && decode_tile(P, sm, idx, n_tiles, t); idx += n_pairs) {
         const int kb0 = t.ks * num_kb / P.ksplit, kb1 = (t.ks + 1) * num_kb / P.ksplit;
         const int a_row = t.m0 + (int)rank * kBM;
-        // bytes both CTAs bring in per stage (a half-width tile of the last round has half the B bytes)
-        const uint32_t tx_pair = 2u * (n_a * a_bytes + (t.bn == P.bn ? b_bytes : b_bytes / 2u));
         int k0 = kb0 * kBK;
         int kB = P.k_wrap > 0 ? k0 % P.k_wrap : k0;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -314,8 +299,8 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           } else if (P.bmode == B_SINGLE) {
             tma_load_4d(st_b, &map_b, kB, P.b_sub, t.n0 + (int)rank * half_bn, t.e, bar);
           } else {
-            const int nc = t.n0 + (int)rank * (t.bn / 2);
-            for (int j = 0; j < t.bn / 128; ++j)
+            const int nc = t.n0 + (int)rank * half_bn;
+            for (int j = 0; j < P.bn / 128; ++j)
               tma_load_4d(st_b + (size_t)j * 64 * kBK * 2, &map_b, nc + 64 * j, P.b_sub, kB, t.e, bar);
           }
           k0 += kBK, kB += kBK;
@@ -334,7 +319,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       // is a counter, not a division, and the operand descriptors are a constant high word plus a low word that
       // steps through the stage (K-major operands: 32 bytes per 16 k-values; N-major: 16 k-rows of 128 bytes).
       const int n_mma = P.bmode == B_PAIR ? 2 * P.bn : P.bn;
-      const uint32_t idesc_full = instr_desc(n_mma, P.bmode == B_NMAJOR), idesc_half = instr_desc(n_mma / 2, P.bmode == B_NMAJOR);
+      const uint32_t idesc = instr_desc(n_mma, P.bmode == B_NMAJOR);
       const uint64_t hi_k = smem_desc(0, 16, 1024) & 0xffffffff00000000ull;
       const uint64_t hi_b = (P.bmode == B_NMAJOR ? smem_desc(0, 64 * kBK * 2, 1024) : smem_desc(0, 16, 1024)) & 0xffffffff00000000ull;
       const uint32_t lo_b_lbo = (P.bmode == B_NMAJOR ? (uint32_t)(64 * kBK * 2 >> 4) : 1u) << 16;
@@ -344,7 +329,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
       uint32_t slot = 0, par = 0, st_lo = stage0;
       int tile_i = 0;
       bool ok = true;
-      for (int idx = pair; ok && decode_tile(P, sm, idx, n_tiles, n_pairs, t); idx += n_pairs, ++tile_i) {
+      for (int idx = pair; ok && decode_tile(P, sm, idx, n_tiles, t); idx += n_pairs, ++tile_i) {
         const int buf = tile_i & 1;
         if (tile_i >= 2) {  // the accumulators two tiles back must have left this buffer, in both CTAs
           if (!mbar_wait(&sm.accum_empty[buf], ((tile_i >> 1) - 1) & 1)) {
@@ -356,7 +341,6 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
         }
         const uint32_t d_tmem = tmem + (uint32_t)(buf * kAccCols);
         const int kb0 = t.ks * num_kb / P.ksplit, kb1 = (t.ks + 1) * num_kb / P.ksplit;
-        const uint32_t idesc = t.bn == P.bn ? idesc_full : idesc_half;
         uint32_t acc = 0;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(&sm.full[slot], par)) {
@@ -393,14 +377,14 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
     const int cpar = (warp - 2) >> 2;  // which of the two warps of this quarter: it takes every other 32-column chunk
     const uint32_t acce_bar[2] = {map_to_rank(&sm.accum_empty[0], 0u), map_to_rank(&sm.accum_empty[1], 0u)};
     int tile_i = 0;
-    for (int idx = pair; decode_tile(P, sm, idx, n_tiles, n_pairs, t); idx += n_pairs, ++tile_i) {
+    for (int idx = pair; decode_tile(P, sm, idx, n_tiles, t); idx += n_pairs, ++tile_i) {
       const int buf = tile_i & 1;
       if (!mbar_wait(&sm.accum_full[buf], (tile_i >> 1) & 1)) {
         if (lane == 0) flag_error(P.st, MOE_ERR_TIMEOUT, 0x402u);
         break;
       }
       tc_fence_after();
-      const int ncols = min(t.bn, P.n_store - t.n0);  // columns of this tile to store (multiple of 8)
+      const int ncols = min(P.bn, P.n_store - t.n0);  // columns of this tile to store (multiple of 8)
       const int row = t.m0 + (int)rank * kBM + 32 * q + lane;
       const bool row_ok = row < t.m_end;
       const uint32_t tbase = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kAccCols);
@@ -454,7 +438,7 @@ __global__ void __launch_bounds__(kThreadsGG, 1)
           }
         }
       } else {
-        for (int c = 32 * cpar; c < t.bn; c += 64) {
+        for (int c = 32 * cpar; c < P.bn; c += 64) {
           uint32_t a[32];
           tc_ld32(tbase + c, a);
           tc_wait_ld();
@@ -638,7 +622,6 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
     if ((rc = make_map_b(&mb, w->gud, d, 3, f, E, 64, kBK)) != MOE_OK) return rc;
     P.K = f, P.n_total = d, P.bn = pick_bn(d, 256, 128), P.bmode = B_NMAJOR, P.b_sub = 2;
     P.epi = EPI_F32, P.out = out_slots, P.ld_out = d, P.out_off2 = 0;
-    P.tail_split = P.bn == 256 ? 1 : 0;
     if (out_planes && n_slots <= kKSplitMaxSlots) {
       // short prefill: too few tiles for the SMs, and every tile streams a long run of weights.  The caller
       // sums planes: cut the contraction so that every pair streams a part, each part into its own plane.
@@ -647,7 +630,6 @@ int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, 
       int ks = (int)((ctx->sm_count / 2) / std::max<long long>(tiles, 1));
       ks = std::min(std::min(ks, kKSplitMax), (f + kBK - 1) / kBK);
       if (ks > 1) {
-        P.tail_split = 0;
         P.ksplit = ks, P.plane_elems = (long long)n_slots * d;
         *out_planes = ks;
       }

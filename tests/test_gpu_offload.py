@@ -163,3 +163,47 @@ def test_expert_replacements_kernel_matches_eq4_and_fig5():
         torch.cuda.synchronize()
         _, H = X.hard_replacements(X.activity_from_topk(S, E))
         assert int(out.item()) == H
+
+
+def test_delta_uniform_kernel_matches_checker():
+    """Expert balance per layer (Section 3.3): integer counts exactly, the deviation from uniform against the
+    checker's reading of it (the paper prints no formula: parity unpinned on both sides)."""
+    from paper_2503_00245_b200 import binding as B
+    for seed, (Bn, T, k, E) in enumerate([(3, 50, 2, 8), (1, 1, 1, 4), (24, 256, 2, 16)]):
+        S = np.stack([W.sticky_routing_trace(300 + seed * 40 + b, T, E, k, 0.5) for b in range(Bn)]).astype(np.int32)
+        counts = torch.zeros((Bn, E), dtype=torch.int64, device="cuda")
+        delta = torch.zeros(Bn + 1, dtype=torch.float64, device="cuda")
+        bad = torch.zeros(1, dtype=torch.int64, device="cuda")
+        B.moe_delta_uniform(torch.from_numpy(S).cuda(), Bn, T, k, E, counts, delta, bad)
+        torch.cuda.synchronize()
+        A = X.activity_from_topk(S, E)
+        assert counts.cpu().numpy().tolist() == A.sum(axis=1).tolist()
+        want = [X.delta_uniform(A[b:b + 1]) for b in range(Bn)]
+        got = delta.cpu().numpy()
+        assert np.allclose(got[:Bn], want, rtol=0, atol=1e-12)
+        assert abs(got[Bn] - float(np.mean(want))) <= 1e-12
+        assert int(bad.item()) == 0
+    # ids outside [0, E) are reported, not counted
+    S = np.int32([[[0, 1], [9, 1], [-1, 0]]])
+    counts = torch.zeros((1, 4), dtype=torch.int64, device="cuda")
+    delta = torch.zeros(2, dtype=torch.float64, device="cuda")
+    bad = torch.zeros(1, dtype=torch.int64, device="cuda")
+    B.moe_delta_uniform(torch.from_numpy(S).cuda(), 1, 3, 2, 4, counts, delta, bad)
+    torch.cuda.synchronize()
+    assert counts.cpu().numpy().tolist() == [[2, 2, 0, 0]] and int(bad.item()) == 2
+
+
+def test_expert_replacements_reads_rows_as_sets():
+    """Eq. 4 is written on the 0/1 activity matrix: a repeated id in a row counts once, an id outside the
+    range not at all."""
+    from paper_2503_00245_b200 import binding as B
+    S = np.int32([[[0, 0], [0, 1], [5, 1], [1, 1], [2, 3]]])      # E = 4: id 5 does not exist
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    B.moe_expert_replacements(torch.from_numpy(S).cuda(), 1, 5, 2, 4, out)
+    torch.cuda.synchronize()
+    A = np.zeros((1, 5, 4), dtype=np.int64)
+    for t, row in enumerate(S[0]):
+        for e in row:
+            if 0 <= e < 4:
+                A[0, t, e] = 1
+    assert int(out.item()) == X.hard_replacements(A)[1]
