@@ -115,6 +115,16 @@ int moe_destroy(moe_ctx* ctx);
 int moe_check(moe_ctx* ctx, void* stream);
 /* Scratch the hot calls need for T tokens (upper bound over all calls and paths). */
 int moe_workspace_bytes(const moe_config* cfg, int32_t T, size_t* bytes);
+/* Diagnostics, for testing the time-out path without hanging or faulting anything.  Not for production use.
+ * moe_set_finaliser_wait: how many SM clock cycles the finalising CTAs of the dense streaming kernel wait for
+ * the other CTAs' partial sums before they give up and flag MOE_ERR_TIMEOUT (0 = the default, about two seconds).
+ * moe_seed_arrival_counter: overwrites the ctx's arrival counter (which normally runs over launches and is a
+ * multiple of the grid size between calls) and waits for `stream`.  Seeded with grid size - 1, the next launch's
+ * arrivals straddle a multiple of the grid size, so most of its finalisers wait for a count that launch never
+ * reaches: with a short budget they give up, every CTA having streamed its share and exited normally.  The
+ * output of such a call is undefined; moe_check reports MOE_ERR_TIMEOUT and re-arms the state.               */
+int moe_set_finaliser_wait(moe_ctx* ctx, long long cycles);
+int moe_seed_arrival_counter(moe_ctx* ctx, unsigned long long value, void* stream);
 /* Kernels launched by hot calls on this ctx since creation (for accounting). */
 int moe_launch_count(moe_ctx* ctx, uint64_t* launches);
 

@@ -49,6 +49,8 @@ _SIGS = {
     "moe_check": (C.c_int, [_P, _P]),
     "moe_workspace_bytes": (C.c_int, [C.POINTER(moe_config), C.c_int32, C.POINTER(C.c_size_t)]),
     "moe_launch_count": (C.c_int, [_P, C.POINTER(C.c_uint64)]),
+    "moe_set_finaliser_wait": (C.c_int, [_P, C.c_longlong]),
+    "moe_seed_arrival_counter": (C.c_int, [_P, C.c_ulonglong, _P]),
     "moe_pack_dense": (C.c_int, [C.c_int32] * 3 + [_P] * 5),
     "moe_pack_wd": (C.c_int, [C.c_int32] * 4 + [_P] * 11),
     "moe_route": (C.c_int, [_P, _P, C.c_int32, C.POINTER(moe_weights), _P, _P, _P, _P]),
@@ -141,6 +143,14 @@ def moe_workspace_bytes(cfg: moe_config, T: int) -> int:
     n = C.c_size_t()
     _ok(_lib().moe_workspace_bytes(C.byref(cfg), T, C.byref(n)), "moe_workspace_bytes")
     return n.value
+
+
+def moe_set_finaliser_wait(ctx: int, cycles: int):
+    _ok(_lib().moe_set_finaliser_wait(ctx, cycles), "moe_set_finaliser_wait")
+
+
+def moe_seed_arrival_counter(ctx: int, value: int, stream=None):
+    _ok(_lib().moe_seed_arrival_counter(ctx, value, _stream(stream)), "moe_seed_arrival_counter")
 
 
 def moe_launch_count(ctx: int) -> int:

@@ -129,6 +129,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out) {
   c->cfg = *cfg;
   c->device = dev;
   c->launches = 0;
+  c->fin_wait_budget = 0;
   c->d_state = nullptr;
   c->h_state = nullptr;
   c->acc = nullptr;
@@ -184,6 +185,22 @@ int moe_workspace_bytes(const moe_config* cfg, int32_t T, size_t* bytes) {
   if (rc != MOE_OK) return rc;
   if (T < 0) return MOE_ERR_INVALID_ARG;
   *bytes = ws_layout(*cfg, T).total;
+  return MOE_OK;
+}
+
+int moe_set_finaliser_wait(moe_ctx* ctx, long long cycles) {
+  if (!ctx || cycles < 0) return MOE_ERR_INVALID_ARG;
+  ctx->fin_wait_budget = cycles;
+  return MOE_OK;
+}
+
+int moe_seed_arrival_counter(moe_ctx* ctx, unsigned long long value, void* stream) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  ctx->h_state->done_total = value;
+  MOE_CUDA_TRY(cudaMemcpyAsync(&ctx->d_state->done_total, &ctx->h_state->done_total, sizeof(unsigned long long),
+                               cudaMemcpyHostToDevice, s));
+  MOE_CUDA_TRY(cudaStreamSynchronize(s));
   return MOE_OK;
 }
 

@@ -54,6 +54,7 @@ struct moe_ctx {
   long long* acc;                // device: fixed-point output accumulators of the dense streaming path, kept zero
   size_t acc_elems;              //         between calls by the kernel itself (MOE_STREAM_MAX_TOKENS*top_k*d)
   unsigned long long launches;
+  long long fin_wait_budget;     // cycles the dense streaming kernel's finalisers wait for the arrival counter (0 = default)
 };
 
 namespace cosmoe {

@@ -62,6 +62,7 @@ struct DenseParams {
   int wpart_ok;                // shared memory holds the [8][d] merge buffer of the unit-owner passes (d <= 1024)
   int acc_copies;              // the CTAs spread their atomics over this many accumulator copies
   long long acc_copy_stride;   // elements between copies
+  long long fin_wait_budget;   // cycles a finalising CTA waits for the arrival counter to fill up
 };
 
 struct Smem {
@@ -1092,7 +1093,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     if (slice >= 0 && old != G - 1u) {
       const long long t0 = clock64();
       while (ld_acquire64(&st->done_total) < target) {
-        if (clock64() - t0 > kWaitBudgetCycles || sm.abort || ld_acquire(&st->status) != 0u) {
+        if (clock64() - t0 > P.fin_wait_budget || sm.abort || ld_acquire(&st->status) != 0u) {
           flag_error(st, MOE_ERR_TIMEOUT, 0x340u);  // (keeps an earlier error code if one is set)
           slice = -1;
           break;
@@ -1187,6 +1188,7 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
     const long long want = rows >= 16 ? 1 : (16 / rows < 8 ? 16 / rows : 8);  // rows x copies of about 16 spread the atomics enough
     P.acc_copies = (int)(fit < want ? fit : want);
   }
+  P.fin_wait_budget = ctx->fin_wait_budget > 0 ? ctx->fin_wait_budget : kWaitBudgetCycles;
   const int xrow = c.d_model * (P.x_is_bf16 ? 2 : 4);
   P.xs_bytes = T > 1 ? ((T * xrow + 1) / 2 + 127) / 128 * 128   // several tokens: the two buffers together hold all rows
                      : (xrow + 127) / 128 * 128;
