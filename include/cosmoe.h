@@ -186,7 +186,10 @@ int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights*
  * before launching, and two calls that overlap on the GPU (different streams, or different threads)
  * race on it -- issue them in one stream or serialise them yourself.
  * T == 0 does no work: it waits for `stream` and returns what the kernels of earlier calls on this GPU
- * reported (MOE_OK, MOE_ERR_TIMEOUT or MOE_ERR_STATE), clearing the report.                          */
+ * reported (MOE_OK, MOE_ERR_TIMEOUT or MOE_ERR_STATE), clearing the report.  Until it is cleared, a
+ * report stays: the kernels of later calls see it and leave their output unwritten, although those
+ * calls return MOE_OK (they only enqueue) -- so poll with T == 0 wherever moe_check would be called.
+ * The one-off set-up is thread-safe; a device that is not sm_100 gets MOE_ERR_NO_DEVICE.              */
 int moe_layer_forward_static(const moe_config* cfg, const void* x, int32_t T, const moe_weights* w, void* y,
                              int32_t* topk_idx, float* topk_w, void* stream);
 

@@ -22,6 +22,8 @@
 // With one token (T == 1, the batch-1 decode case) the router runs in the prologue of every CTA
 // (logits, softmax, top-k, gate weights: Eq. 2, Eq. 3), so the layer is a single launch.
 // Every wait is bounded; an expired wait sets the ctx's status word and the kernel winds down.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace cosmoe {
@@ -1244,24 +1246,32 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 
 constexpr int kMaxDevices = 64;
 struct StaticDevice {
-  int ready;
+  std::once_flag once;
+  int rc;               // outcome of the one-off set-up
   unsigned char* base;  // device address of g_static_scratch on this GPU
   int sm_count, max_smem_optin;
 };
 StaticDevice g_static_dev[kMaxDevices];
 
-// Once per device, with that device current: resolve the array's device address.
+int static_setup_once(int dev, StaticDevice& sd) {
+  int major = 0;
+  void* p = nullptr;
+  MOE_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (major != 10) return MOE_ERR_NO_DEVICE;  // kernels are built for sm_100a only
+  MOE_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+  MOE_CUDA_TRY(cudaDeviceGetAttribute(&sd.sm_count, cudaDevAttrMultiProcessorCount, dev));
+  MOE_CUDA_TRY(cudaDeviceGetAttribute(&sd.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  sd.base = (unsigned char*)p;
+  return MOE_OK;
+}
+
+// Once per device, with that device current: resolve the array's device address.  Safe to reach from several
+// threads at once (std::call_once orders the set-up before every caller's use of its results).
 int static_setup(int dev, StaticDevice** out) {
   if (dev < 0 || dev >= kMaxDevices) return MOE_ERR_UNSUPPORTED;
   StaticDevice& sd = g_static_dev[dev];
-  if (!sd.ready) {
-    void* p = nullptr;
-    MOE_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
-    MOE_CUDA_TRY(cudaDeviceGetAttribute(&sd.sm_count, cudaDevAttrMultiProcessorCount, dev));
-    MOE_CUDA_TRY(cudaDeviceGetAttribute(&sd.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    sd.base = (unsigned char*)p;
-    sd.ready = 1;
-  }
+  std::call_once(sd.once, [&] { sd.rc = static_setup_once(dev, sd); });
+  if (sd.rc != MOE_OK) return sd.rc;
   *out = &sd;
   return MOE_OK;
 }

@@ -29,7 +29,15 @@ def _pair(sh, T, step):
     return B, lay, x, ref, y, idx, w
 
 
-@pytest.mark.parametrize("sh,T", [(W.WEARABLE, 1), (W.WEARABLE, 8), (W.TINY, 16)])
+E6 = W.LayerShape("six experts", 8, 136, 200, n_experts=6, top_k=3)
+
+
+@pytest.mark.parametrize("sh,T", [
+    (W.WEARABLE, 1), (W.WEARABLE, 8), (W.TINY, 16),
+    (W.PHONE, 1),     # d_model at the limit
+    (W.PHONE, 16),    # d_model and T at the limit: the accumulators fill the scratch array exactly
+    (E6, 5),          # E not 8 or 16 with several tokens: the router runs as its own kernel first
+])
 def test_static_entry_matches_ordinary_entry_twice_in_a_row(sh, T):
     for step in (1, 2):                       # two calls in a row, different inputs
         B, lay, x, ref, y, idx, w = _pair(sh, T, step)
@@ -57,3 +65,29 @@ def test_static_entry_rejects_what_does_not_fit():
     assert B.moe_layer_forward_static(wd, t["x"], 1, lay.weights, y) == 2             # decomposed experts
     assert B.moe_layer_forward_static(lay.cfg, t["x"], 16, lay.weights, y) == 1       # T > 1 without routing buffers
     lay.close()
+
+
+def test_static_entry_single_token_without_routing_buffers_and_against_the_checker():
+    """T == 1 with topk_idx / topk_w NULL, twice in a row; the second output also against the CPU checker."""
+    from paper_2503_00245_b200 import binding as B
+    sh = W.WEARABLE
+    lay, t, host = U.build(sh, 1, path=B.MOE_PATH_STREAM)
+    for step in (3, 4):
+        x = W.make_x(sh, 1, device="cuda", step=step)
+        ref = lay.forward(x)
+        y = torch.full_like(x, float("nan"))
+        assert B.moe_layer_forward_static(lay.cfg, x, 1, lay.weights, y) == 0
+        torch.cuda.synchronize()
+        assert B.moe_layer_forward_static(lay.cfg, x, 0, lay.weights, y) == 0
+        assert torch.equal(y, ref)
+    h = dict(host)
+    h["x"] = W.to_host_bits(x)
+    ora = U.oracle_layer(h, sh.top_k)
+    if not O_near(ora, sh.top_k).any():
+        U.assert_close_rms(U.to64(y), ora["y"])
+    lay.close()
+
+
+def O_near(ora, k):
+    from oracle import moe_oracle as O
+    return O.near_tie_tokens(ora["logits"], k, U.TIE_GAP)
