@@ -217,13 +217,18 @@ int moe_offload_slot_table(moe_offload* off, int32_t layer, const int32_t** expe
 int moe_offload_resident(moe_offload* off, int32_t layer, int32_t* slots_host);
 int moe_offload_stats(moe_offload* off, uint64_t* fetches, uint64_t* bytes, uint64_t* hits);
 
-/* One decode step (T = 1) through n_layers stacked MoE layers with offloaded
- * experts: per layer u = h / rms(h), route(u) -> routing read back to the host ->
- * moe_offload_ensure -> y = experts(u) with the gate weights -> h += y.
- * h dev [d] fp32, updated in place.  routers: host array of n_layers moe_weights whose
- * w_router / b_router are set (expert pointers are taken from the offload object).
- * topk_trace_host [n_layers][k] receives each layer's selection.  Synchronises
- * `stream` once per layer (the host must see the routing before it can copy).      */
+/* One decode step (T = 1) through n_layers stacked MoE layers with offloaded experts.  Per layer:
+ * u = h / rms(h) (no learned scale) rounded to cfg.x_dtype, the router on u, y = experts(u) with the gate
+ * weights, h += y (fp32, y not rounded in between).  h dev [d] fp32, updated in place.  routers: host array of
+ * n_layers moe_weights whose w_router / b_router are set (expert pointers are taken from the offload object).
+ * topk_trace_host [n_layers][k] receives each layer's selection.
+ * The host must see a layer's selection before it can copy: a small kernel (norm + router) writes it to mapped
+ * pinned memory and the host polls for it (bounded: MOE_ERR_TIMEOUT after 10 s) -- no stream synchronisation.
+ * Overlap: the resident selected experts of the layer run at once; a missing expert is copied in chunks of about
+ * 8 MB on the offload's copy stream, and the launch that computes a chunk's hidden units waits only for that
+ * chunk, so compute trails the copy by one chunk and the link goes idle only between the last chunk of a layer
+ * and the routing of the next.  All launches of a layer add into the ctx's fixed-point accumulators; the last
+ * converts them.  Returns with the work queued; wait for `stream` (or call moe_check) before reading h.     */
 int moe_stack_decode_step(moe_offload* off, moe_ctx* ctx, const moe_weights* routers, float* h,
                           int32_t* topk_trace_host, void* ws, size_t ws_bytes, void* stream);
 
@@ -232,10 +237,14 @@ int moe_stack_decode_step(moe_offload* off, moe_ctx* ctx, const moe_weights* rou
  * the router's probabilities (Eq. 2) of those experts, renormalised over the set.  For
  * replaying routing traces, e.g. traces with a given expert replacement ratio (Eq. 4-5)
  * under the rule of Eq. 8.  Because the host knows the sets, it does not wait for the
- * device between layers: a layer's misses are copied on the offload's copy stream while
- * earlier layers compute.  Synchronises `stream` once, at the end.                      */
+ * device at all: a layer's misses are copied on the offload's copy stream while earlier layers
+ * compute, and a layer is ONE launch (norm, router, experts, residual add).  Returns with the work queued. */
 int moe_stack_decode_step_trace(moe_offload* off, moe_ctx* ctx, const moe_weights* routers, float* h,
                                 const int32_t* sel_host, void* ws, size_t ws_bytes, void* stream);
+
+/* Host wall time moe_stack_decode_step has spent so far waiting for routing words (poll_s, over `polls`
+ * waits) and queueing copies and launches (issue_s): where a token's time goes besides the link.        */
+int moe_offload_host_times(moe_offload* off, double* poll_s, double* issue_s, uint64_t* polls);
 
 /* ---- routing-trace metrics (Eq. 4-5, Section 2.3 / 3.3) ---------------------------
  * topk_trace dev [B][T][k] int32.  Writes H (Eq. 4, summed over experts) to

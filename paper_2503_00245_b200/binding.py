@@ -69,6 +69,7 @@ _SIGS = {
     "moe_stack_decode_step": (C.c_int, [_P, _P, C.POINTER(moe_weights), _P, C.POINTER(C.c_int32), _P, C.c_size_t, _P]),
     "moe_stack_decode_step_trace": (C.c_int, [_P, _P, C.POINTER(moe_weights), _P, C.POINTER(C.c_int32), _P, C.c_size_t,
                                               _P]),
+    "moe_offload_host_times": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_uint64)]),
     "moe_expert_replacements": (C.c_int, [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P]),
     "moe_delta_uniform": (C.c_int, [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P]),
 }
@@ -265,3 +266,9 @@ def moe_expert_replacements(topk_trace, B, T, k, n_experts, h_total_out, stream=
 def moe_delta_uniform(topk_trace, B, T, k, n_experts, counts_out, delta_out, bad_out, stream=None):
     _ok(_lib().moe_delta_uniform(_ptr(topk_trace), B, T, k, n_experts, _ptr(counts_out), _ptr(delta_out),
                                  _ptr(bad_out), _stream(stream)), "moe_delta_uniform")
+
+
+def moe_offload_host_times(off: int):
+    a, b, n = C.c_double(), C.c_double(), C.c_uint64()
+    _ok(_lib().moe_offload_host_times(off, C.byref(a), C.byref(b), C.byref(n)), "moe_offload_host_times")
+    return {"poll_s": a.value, "issue_s": b.value, "polls": n.value}

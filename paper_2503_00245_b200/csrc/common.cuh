@@ -96,10 +96,21 @@ int launch_stream_ffn(moe_ctx* ctx, int mode, const void* x, int T, const moe_we
                       char* ws, const WsLayout& L, cudaStream_t s);
 // Dense experts, streaming path, one kernel (router fused when T == 1 and mode == 0; mode 2 = mode 0 with the
 // routing always taken from topk_idx / topk_w).
+// Optional extras of a single-token launch of the dense streaming kernel (the stacked decode steps use them).
+struct DenseExtra {
+  unsigned sel_mask;                 // routing given: which of the k routing entries this launch computes (0 = all)
+  int slot_of_entry[MOE_MAX_TOPK];   // slot of the packed array that holds routing entry j's expert (-1: expert_slot table)
+  int unit_lo, unit_cnt;             // hidden units [unit_lo, unit_lo + unit_cnt) of every expert only (unit_cnt 0 = all)
+  int finalize;                      // 0: leave the partial sums in the accumulators for a later launch of the group
+  float* resid;                      // fp32 [d]: the finalisers add the layer's output to it (h += y) instead of writing y
+  const float* h_in;                 // fp32 [d]: the layer input is h / rms(h), computed in the prologue (router fused)
+  int use_forced;                    // router fused: the expert set is prescribed, the gate weights are its probabilities
+  int forced[MOE_MAX_TOPK];
+};
 bool dense_stream_fuses_route(const moe_config& c, int T);  // mode 0 computes the routing itself (else: run launch_route first)
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
                         float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
-                        cudaStream_t s);
+                        cudaStream_t s, const DenseExtra* ex = nullptr);
 // Tensor-core (prefill) path: out_slots from x gathered by perm.
 int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, const int32_t* offsets,
                       const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, int* out_planes,
@@ -358,6 +369,32 @@ __device__ __forceinline__ void warp_route_finish(float l0, float l1, int E, int
     const float pw = expf(f32_unkey(best) - m) * inv_sum;
     wtot += pw;
     if (lane == j) my_w = pw, my_idx = win;
+  }
+  if (lane < k) {
+    idx_out[lane] = my_idx;
+    w_out[lane] = renorm ? my_w / wtot : my_w;
+  }
+}
+
+// The same with the expert set prescribed (sel[0..k), distinct): the gate weights are the softmax probabilities
+// (Eq. 2) of those experts, renormalised over the set when `renorm`.  Lane j < k writes the j-th entry.
+__device__ __forceinline__ void warp_route_forced(float l0, float l1, int E, int k, int renorm, int lane,
+                                                  const int* __restrict__ sel, int32_t* __restrict__ idx_out,
+                                                  float* __restrict__ w_out) {
+  const unsigned FULL = 0xffffffffu;
+  const float NEG = -3.402823466e38f;
+  const bool has0 = lane < E, has1 = lane + 32 < E;
+  const float m = f32_unkey(__reduce_max_sync(FULL, f32_key(fmaxf(has0 ? l0 : NEG, has1 ? l1 : NEG))));
+  const float p0 = has0 ? expf(l0 - m) : 0.f, p1 = has1 ? expf(l1 - m) : 0.f;
+  const float inv_sum = 1.0f / warp_sum(p0 + p1);
+  float my_w = 0.f, wtot = 0.f;
+  int my_idx = 0;
+  for (int j = 0; j < k; ++j) {
+    const int e = sel[j];
+    const float a = __shfl_sync(FULL, p0, e & 31), b = __shfl_sync(FULL, p1, e & 31);
+    const float pw = (e < 32 ? a : b) * inv_sum;
+    wtot += pw;
+    if (lane == j) my_w = pw, my_idx = e;
   }
   if (lane < k) {
     idx_out[lane] = my_idx;

@@ -65,6 +65,9 @@ struct DenseParams {
   int acc_copies;              // the CTAs spread their atomics over this many accumulator copies
   long long acc_copy_stride;   // elements between copies
   long long fin_wait_budget;   // cycles a finalising CTA waits for the arrival counter to fill up
+  int f_full;                  // hidden units per expert in memory (f may be a sub-range of them, starting at ex.unit_lo)
+  int given1;                  // one token, routing taken from topk_idx / topk_w (possibly a subset of its entries)
+  DenseExtra ex;
 };
 
 struct Smem {
@@ -667,7 +670,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     sm.last = 0;
     sm.zero16[0] = sm.zero16[1] = sm.zero16[2] = sm.zero16[3] = 0u;
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (fused1) {
+    if (fused1 && !P.ex.h_in) {
       // one token: every pass reads token row 0, so the first pass's copy of x can start before the routing
       const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
       mbar_arrive_expect_tx(&sm.xfull[0], xrow_bytes);
@@ -693,6 +696,43 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       wr0[j] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + j * kConsumerThreads, P.d - 1) * P.E));
   }
   if (tid != kConsumerThreads) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Stacked decode: the layer input is u = h / rms(h) (fp32 h, no learned scale), formed here by every CTA, rounded
+  // to the type of x, kept in shared memory as token row 0 and used for the router below.
+  const bool from_h = fused1 && P.ex.h_in != nullptr;
+  if (from_h) {
+    float* rsum = &sm.red[0][0][0][0];
+    float hv[kRJ];
+    float ss = 0.f;
+    if (warp < kWarps) {
+#pragma unroll
+      for (int j = 0; j < kRJ; ++j) {
+        const int i = tid + j * kConsumerThreads;
+        hv[j] = i < P.d ? P.ex.h_in[i] : 0.f;
+        ss = fmaf(hv[j], hv[j], ss);
+      }
+      ss = warp_sum(ss);
+      if (lane == 0) rsum[warp] = ss;
+    }
+    __syncthreads();
+    if (warp < kWarps) {
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) tot += rsum[w];
+      const float inv = rsqrtf(tot / (float)P.d);
+#pragma unroll
+      for (int j = 0; j < kRJ; ++j) {
+        const int i = tid + j * kConsumerThreads;
+        if (i < P.d) {
+          if (P.x_is_bf16)
+            reinterpret_cast<__nv_bfloat16*>(xs)[i] = __float2bfloat16_rn(hv[j] * inv);
+          else
+            reinterpret_cast<float*>(xs)[i] = hv[j] * inv;
+        }
+      }
+    }
+  }
+  // (each thread reads back only the elements it wrote itself: no barrier needed before the router)
+  const void* const xsrc = from_h ? (const void*)xs : P.x;
   if (fused1) {
     // router logits of the single token: every consumer thread takes rows of W_r (row i = the E weights
     // of input feature i), 8 experts at a time
@@ -704,7 +744,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
 #pragma unroll
         for (int j = 0; j < kRJ; ++j) {
           const int i = min(tid + j * kConsumerThreads, d - 1);
-          xv[j] = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[i]) : ((const float*)P.x)[i];
+          xv[j] = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)xsrc)[i]) : ((const float*)xsrc)[i];
           if (tid + j * kConsumerThreads >= d) xv[j] = 0.f;
         }
         for (int e8 = 0; e8 < E; e8 += 8) {
@@ -734,7 +774,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         for (int e = 0; e < E; ++e) {
           float a = 0.f;
           for (int i = tid; i < d; i += kConsumerThreads) {
-            const float xv = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)P.x)[i]) : ((const float*)P.x)[i];
+            const float xv = P.x_is_bf16 ? bf16_to_float(((const uint16_t*)xsrc)[i]) : ((const float*)xsrc)[i];
             a = fmaf(xv, bf16_to_float(__ldg(P.w_router + (size_t)i * E + e)), a);
           }
           a = warp_sum(a);
@@ -748,20 +788,26 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       if (lane + 32 < P.E) bias1 = P.b_router[lane + 32];
     }
     __syncthreads();
+    // token row 0 was written by the consumer threads (input formed from h): it counts as landed
+    if (from_h && tid == kConsumerThreads) mbar_arrive(&sm.xfull[0]);
     if (warp == 0) {
       float l0 = bias0, l1 = bias1;
       if (lane < P.E)
         for (int w = 0; w < kWarps; ++w) l0 += sm.rlog[w][lane];
       if (lane + 32 < P.E)
         for (int w = 0; w < kWarps; ++w) l1 += sm.rlog[w][lane + 32];
-      warp_route_finish(l0, l1, P.E, P.k, P.renorm, lane, sm.stage_e, sm.stage_w, nullptr);
+      if (P.ex.use_forced)
+        warp_route_forced(l0, l1, P.E, P.k, P.renorm, lane, P.ex.forced, sm.stage_e, sm.stage_w);
+      else
+        warp_route_finish(l0, l1, P.E, P.k, P.renorm, lane, sm.stage_e, sm.stage_w, nullptr);
       __syncwarp();
       // the k selected experts in ascending order are the active experts, one slot (token 0) each
       if (lane < P.k) {
         const int e = sm.stage_e[lane];
         int rank = 0;
         for (int i = 0; i < P.k; ++i) rank += (sm.stage_e[i] < e);
-        const int sl = P.expert_slot ? P.expert_slot[e] : e;
+        const int given = P.ex.slot_of_entry[lane];  // the host may know the slot (offload cache)
+        const int sl = given >= 0 ? given : (P.expert_slot ? P.expert_slot[e] : e);
         if (sl < 0) flag_error(st, MOE_ERR_STATE, 0x301u);
         sm.act_e[rank] = e;
         sm.act_slot[rank] = sl < 0 ? 0 : sl;
@@ -848,6 +894,37 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
       }
     }
+  } else if (P.given1) {
+    // one token, routing given: the entries of topk_idx / topk_w this launch was asked for, ascending by expert
+    if (warp == 0) {
+      const bool mine = lane < P.k && ((P.ex.sel_mask >> lane) & 1u);
+      int e = mine ? P.topk_idx[lane] : -1;
+      const float wv = mine ? P.topk_w[lane] : 0.f;
+      int bad = mine && (e < 0 || e >= P.E);
+      if (bad) e = -1;
+      int rank = 0;
+      for (int i = 0; i < P.k; ++i) {
+        const int ei = __shfl_sync(0xffffffffu, e, i);
+        rank += (ei >= 0 && ei < e);
+      }
+      const int na = __popc(__ballot_sync(0xffffffffu, e >= 0));
+      if (e >= 0) {
+        const int given = P.ex.slot_of_entry[lane];
+        const int sl = given >= 0 ? given : (P.expert_slot ? P.expert_slot[e] : e);
+        bad |= sl < 0;
+        sm.act_e[rank] = e;
+        sm.act_slot[rank] = sl < 0 ? 0 : sl;
+        sm.act_off[rank] = rank;
+        sm.slot_tok[rank] = 0;
+        sm.slot_w[rank] = wv;
+      }
+      bad = __any_sync(0xffffffffu, bad);
+      if (lane == 0) {
+        sm.act_off[bad ? 0 : na] = bad ? 0 : na;
+        sm.n_act = bad ? 0 : na;
+        if (bad) flag_error(st, MOE_ERR_STATE, 0x302u);
+      }
+    }
   } else if (P.mode == 0 && warp == 0) {
     for (int p = lane; p < n_pairs; p += 32) {
       sm.stage_e[p] = P.topk_idx[p];
@@ -855,7 +932,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     }
   }
   __syncthreads();
-  if (warp == 0 && !fused1 && P.mode == 0) {
+  if (warp == 0 && !fused1 && !P.given1 && P.mode == 0) {
     // routing products -> active experts and their slots (same numbering as moe_permute): lane e works for
     // experts e and e + 32
     const int n = n_pairs, E = P.E;
@@ -1003,7 +1080,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
                    (const unsigned char*)P.x + (size_t)sm.slot_tok[slot0 + s] * xrow_bytes, xrow_bytes, &sm.xfull[b]);
       }
       const unsigned char* src = reinterpret_cast<const unsigned char*>(P.gud) +
-                                 ((size_t)sm.act_slot[ps.ai] * P.f + ps.ra) * row_bytes;
+                                 ((size_t)sm.act_slot[ps.ai] * P.f_full + P.ex.unit_lo + ps.ra) * row_bytes;
       for (int row = ps.ra; row < ps.rb; row += kRows) {
         const uint32_t bytes = (uint32_t)min(kRows, ps.rb - row) * row_bytes;
         if (rp.n >= NS) {
@@ -1081,6 +1158,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   // (after an expired wait the warps may be out of step with this barrier: then it can expire too; the
   // status word is already set and nobody finalises)
   bool fin = consumer_sync(sm, cpar, lane);
+  if (!P.ex.finalize) return;  // a later launch of the group adds its share and finalises
   // The last kFinalizers CTAs to arrive turn the fixed-point sums into the output, one slice each, and leave
   // zeros behind.  All but the very last of them first wait (bounded) for the arrival counter to fill up: the
   // CTAs they wait for are running or can start on the SMs the finished ones have left.
@@ -1137,6 +1215,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         const float fv = (float)((double)v * kFixInv);
         if (P.mode == 1)
           P.out_slots[i] = fv;
+        else if (P.ex.resid)
+          P.ex.resid[i] += fv;  // h += y (one token; exactly one thread of one CTA owns element i)
         else if (P.x_is_bf16)
           ((__nv_bfloat16*)P.y)[i] = __float2bfloat16_rn(fv);
         else
@@ -1168,7 +1248,7 @@ bool dense_stream_fuses_route(const moe_config& c, int T) {
 
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
                         float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
-                        cudaStream_t s) {
+                        cudaStream_t s, const DenseExtra* ex) {
   const moe_config& c = ctx->cfg;
   if (c.d_model > 32 * 8 * kXIters || !ctx->acc) return MOE_ERR_UNSUPPORTED;
   const bool routing_given = (mode == 2);  // mode 2: the whole layer, but with the caller's routing even at T == 1
@@ -1181,6 +1261,22 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   P.topk_idx = topk_idx, P.topk_w = topk_w, P.offsets = offsets, P.perm = perm;
   P.expert_slot = w->expert_slot, P.gud = (const uint16_t*)w->gud;
   P.y = y, P.out_slots = out_slots, P.st = ctx->d_state, P.acc = ctx->acc;
+  P.f_full = c.d_ff;
+  for (int j = 0; j < MOE_MAX_TOPK; ++j) P.ex.slot_of_entry[j] = -1;
+  P.ex.sel_mask = 0xffffffffu, P.ex.finalize = 1;
+  if (ex) {
+    if (T != 1 || mode == 1) return MOE_ERR_INVALID_ARG;
+    if ((ex->h_in || ex->use_forced) && !P.fused_route) return MOE_ERR_INVALID_ARG;
+    P.ex = *ex;
+    if (P.ex.sel_mask == 0u) P.ex.sel_mask = 0xffffffffu;
+    if (P.ex.unit_cnt > 0) {
+      if (P.ex.unit_lo < 0 || P.ex.unit_lo + P.ex.unit_cnt > c.d_ff) return MOE_ERR_INVALID_ARG;
+      P.f = P.ex.unit_cnt;
+    } else {
+      P.ex.unit_lo = 0;
+    }
+  }
+  P.given1 = (mode == 0 && T == 1 && !P.fused_route) ? 1 : 0;
   {
     // contended atomics on few lines are slow: with room in the accumulator buffer, CTAs use up to 8 copies
     const long long rows = (mode == 0) ? T : (long long)T * c.top_k;

@@ -8,6 +8,9 @@
 // Copies run on the object's own stream: it first waits for the compute stream (nobody may still be reading
 // the victim's slot), copies the expert in chunks, updates the layer's expert->slot table in stream order, and
 // the compute stream then waits for the copy stream's event.
+#include <algorithm>
+#include <atomic>
+#include <chrono>
 #include <new>
 #include <vector>
 
@@ -27,30 +30,24 @@ struct moe_offload {
   std::vector<std::vector<int>> slot_of;    // per layer: expert -> slot or -1
   int32_t* d_tables;                        // device [n_layers][E]
   int32_t* h_tables;                        // pinned  [n_layers][E]
-  int32_t* h_route;                         // pinned  [k] routing read-back of the stacked step
+  int32_t* h_route;                         // pinned, mapped: [0..k) the routing of the current layer, [k] its sequence number
+  int32_t* h_route_dev;                     // the same memory as the device sees it
+  int32_t route_seq;                        // sequence number the next routing kernel writes
+  std::vector<cudaEvent_t> chunk_ev;        // one per chunk of the misses of a layer: recorded on the copy stream
+  std::vector<int> chunk_row;               // a missing expert is copied (and computed) in runs of hidden units
+  int n_chunks;                             // [chunk_row[c], chunk_row[c+1]): halves of what is left, so that few copies are
+                                            // issued and the compute that trails the last one is short
   uint64_t fetches, bytes, hits;
+  // what the routed step spent where, summed over its calls (host wall time, seconds)
+  double t_poll, t_issue;
+  uint64_t polls;
 };
 
 namespace cosmoe {
 namespace {
 
-constexpr size_t kCopyChunk = 8u << 20;  // host->device copies are issued in chunks of this size
-
-// A prescribed expert set for one token: the gate weights are the router's probabilities of those experts,
-// renormalised over the set (what the layer computes when it is told which experts to use).
-struct ForcedSel {
-  int32_t e[MOE_MAX_TOPK];
-};
-__global__ void forced_routing_kernel(const float* __restrict__ probs, int k, int renorm, ForcedSel f,
-                                      int32_t* __restrict__ idx, float* __restrict__ wt) {
-  const int lane = threadIdx.x;
-  const float p = lane < k ? probs[f.e[lane]] : 0.f;
-  const float sum = warp_sum(p);
-  if (lane < k) {
-    idx[lane] = f.e[lane];
-    wt[lane] = renorm ? p / sum : p;
-  }
-}
+constexpr size_t kCopyChunk = 8u << 20;  // moe_offload_ensure issues its host->device copies in chunks of this size
+constexpr size_t kLastChunk = 4u << 20;  // stacked steps: a miss is copied in halves of the rest, down to about this size
 
 // A layer's expert -> slot table, passed BY VALUE: every queued update carries its own copy, so a later call
 // for the same layer cannot change what an earlier, still pending update writes.
@@ -61,29 +58,90 @@ __global__ void slot_table_kernel(int32_t* __restrict__ table, int E, SlotTable 
   if ((int)threadIdx.x < E) table[threadIdx.x] = t.slot[threadIdx.x];
 }
 
-// u = h / sqrt(mean(h^2)) -> x (bf16 or fp32); one CTA
-__global__ void rms_glue_kernel(const float* __restrict__ h, int d, void* __restrict__ x, int x_is_bf16) {
-  __shared__ float s_part[32];
-  float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) ss = fmaf(h[i], h[i], ss);
+// Stacked decode, routed: u = h / rms(h) rounded to the type of x, the router on u (Eq. 2, Eq. 3), and the
+// selection handed to the host through mapped pinned memory: the k expert ids, a system-scope fence, then the
+// sequence number the host polls for.  One CTA; thread t takes the input features t, t + 256, ...
+constexpr int kRouteThreads = 256;
+constexpr int kRouteFeat = 8;  // features per thread: d <= 2048
+__global__ void __launch_bounds__(kRouteThreads)
+    rms_route_kernel(const float* __restrict__ h, int d, int E, int k, int renorm, const uint16_t* __restrict__ w_router,
+                     const float* __restrict__ bias, void* __restrict__ u, int x_is_bf16, int32_t* __restrict__ idx,
+                     float* __restrict__ wt, volatile int32_t* __restrict__ host_route, int32_t seq) {
+  __shared__ float s_sum[kRouteThreads / 32];
+  __shared__ float s_log[kRouteThreads / 32][MOE_MAX_EXPERTS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float hv[kRouteFeat], ss = 0.f;
+#pragma unroll
+  for (int j = 0; j < kRouteFeat; ++j) {
+    const int i = tid + j * kRouteThreads;
+    hv[j] = i < d ? h[i] : 0.f;
+    ss = fmaf(hv[j], hv[j], ss);
+  }
   ss = warp_sum(ss);
-  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+  if (lane == 0) s_sum[warp] = ss;
   __syncthreads();
   float tot = 0.f;
-  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += s_part[w];
+#pragma unroll
+  for (int w = 0; w < kRouteThreads / 32; ++w) tot += s_sum[w];
   const float inv = rsqrtf(tot / (float)d);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float v = h[i] * inv;
-    if (x_is_bf16)
-      ((__nv_bfloat16*)x)[i] = __float2bfloat16_rn(v);
-    else
-      ((float*)x)[i] = v;
+#pragma unroll
+  for (int j = 0; j < kRouteFeat; ++j) {
+    const int i = tid + j * kRouteThreads;
+    float v = hv[j] * inv;
+    if (x_is_bf16) {
+      const __nv_bfloat16 b = __float2bfloat16_rn(v);
+      if (i < d) reinterpret_cast<__nv_bfloat16*>(u)[i] = b;
+      v = __bfloat162float(b);  // the router sees what the experts see
+    } else if (i < d) {
+      reinterpret_cast<float*>(u)[i] = v;
+    }
+    hv[j] = i < d ? v : 0.f;
   }
-}
-// h += y
-__global__ void residual_kernel(float* __restrict__ h, const void* __restrict__ y, int d, int y_is_bf16) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < d) h[i] += y_is_bf16 ? __bfloat162float(((const __nv_bfloat16*)y)[i]) : ((const float*)y)[i];
+  for (int e0 = 0; e0 < E; e0 += 8) {
+    float a[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) a[q] = 0.f;
+    if ((E & 7) == 0) {
+#pragma unroll
+      for (int j = 0; j < kRouteFeat; ++j) {
+        const int i = min(tid + j * kRouteThreads, d - 1);
+        float w[8];
+        unpack8(__ldg(reinterpret_cast<const uint4*>(w_router + (size_t)i * E + e0)), w);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) a[q] = fmaf(hv[j], w[q], a[q]);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < kRouteFeat; ++j) {
+        const int i = min(tid + j * kRouteThreads, d - 1);
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          if (e0 + q < E) a[q] = fmaf(hv[j], bf16_to_float(__ldg(w_router + (size_t)i * E + e0 + q)), a[q]);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float t = warp_sum(a[q]);
+      if (lane == 0 && e0 + q < E) s_log[warp][e0 + q] = t;
+    }
+  }
+  __syncthreads();
+  if (warp != 0) return;
+  float l0 = 0.f, l1 = 0.f;
+  if (lane < E) {
+    for (int w = 0; w < kRouteThreads / 32; ++w) l0 += s_log[w][lane];
+    if (bias) l0 += bias[lane];
+  }
+  if (lane + 32 < E) {
+    for (int w = 0; w < kRouteThreads / 32; ++w) l1 += s_log[w][lane + 32];
+    if (bias) l1 += bias[lane + 32];
+  }
+  warp_route_finish(l0, l1, E, k, renorm, lane, idx, wt, nullptr);
+  __syncwarp();
+  if (lane < k) host_route[lane] = idx[lane];
+  __threadfence_system();
+  __syncwarp();
+  if (lane == 0) host_route[k] = seq;
 }
 
 // Eq. 4: H = sum_b sum_t sum_e |[e in S(b,t+1)] - [e in S(b,t)]| = size of the symmetric difference of
@@ -184,14 +242,35 @@ int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_pe
   o->slot_bytes = slot_bytes;
   o->fetches = o->bytes = o->hits = 0;
   o->copy_stream = nullptr, o->ev_compute = nullptr, o->ev_copy = nullptr;
-  o->d_tables = nullptr, o->h_tables = nullptr, o->h_route = nullptr;
+  o->d_tables = nullptr, o->h_tables = nullptr, o->h_route = nullptr, o->h_route_dev = nullptr;
+  o->route_seq = 0, o->t_poll = o->t_issue = 0.0, o->polls = 0;
+  {
+    const size_t row_bytes = (size_t)3 * cfg->d_model * 2;
+    const int min_rows = (int)std::max<size_t>(1, kLastChunk / row_bytes);
+    o->chunk_row.assign(1, 0);
+    for (int left = cfg->d_ff; left > 0;) {
+      const int take = left <= 2 * min_rows ? left : left / 2;
+      o->chunk_row.push_back(o->chunk_row.back() + take);
+      left -= take;
+    }
+    o->n_chunks = (int)o->chunk_row.size() - 1;
+  }
   const size_t tb = (size_t)n_layers * o->E * sizeof(int32_t);
   cudaError_t e = cudaStreamCreateWithFlags(&o->copy_stream, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&o->ev_compute, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&o->ev_copy, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMalloc((void**)&o->d_tables, tb);
   if (e == cudaSuccess) e = cudaMallocHost((void**)&o->h_tables, tb);
-  if (e == cudaSuccess) e = cudaMallocHost((void**)&o->h_route, sizeof(int32_t) * MOE_MAX_TOPK);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&o->h_route, sizeof(int32_t) * (MOE_MAX_TOPK + 1), cudaHostAllocMapped);
+  if (e == cudaSuccess) {
+    for (int j = 0; j <= MOE_MAX_TOPK; ++j) o->h_route[j] = -1;
+    e = cudaHostGetDevicePointer((void**)&o->h_route_dev, o->h_route, 0);
+  }
+  if (e == cudaSuccess) {
+    o->chunk_ev.assign((size_t)cfg->top_k * o->n_chunks, nullptr);
+    for (size_t i = 0; i < o->chunk_ev.size() && e == cudaSuccess; ++i)
+      e = cudaEventCreateWithFlags(&o->chunk_ev[i], cudaEventDisableTiming);
+  }
   if (e == cudaSuccess) {
     o->layer_done.assign(n_layers, nullptr);
     o->layer_done_set.assign(n_layers, 0);
@@ -233,6 +312,8 @@ int moe_offload_destroy(moe_offload* o) {
   if (o->ev_copy) cudaEventDestroy(o->ev_copy);
   for (cudaEvent_t ev : o->layer_done)
     if (ev) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : o->chunk_ev)
+    if (ev) cudaEventDestroy(ev);
   if (o->d_tables) cudaFree(o->d_tables);
   if (o->h_tables) cudaFreeHost(o->h_tables);
   if (o->h_route) cudaFreeHost(o->h_route);
@@ -241,21 +322,28 @@ int moe_offload_destroy(moe_offload* o) {
   return MOE_OK;
 }
 
-// by_layer_event: the caller is a stacked step, which records layer_done[layer] after the layer's kernels
-static int ensure_impl(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, void* compute_stream,
-                       bool by_layer_event) {
-  if (!o || !sel || layer < 0 || layer >= o->n_layers || n <= 0 || n > o->slots) return MOE_ERR_INVALID_ARG;
+// What a layer has to do for one step's selection: per selected expert its slot and whether it must be fetched.
+struct LayerPlan {
+  int n, n_miss;
+  int e[MOE_MAX_TOPK], slot[MOE_MAX_TOPK];
+  bool miss[MOE_MAX_TOPK];
+};
+
+// Bookkeeping only (host integers): hits touch the recency list, a miss takes the slot of the least recently
+// used resident expert that is not selected in this step.  Nothing is queued.
+static int plan_layer(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, LayerPlan& pl) {
+  if (!o || !sel || layer < 0 || layer >= o->n_layers || n <= 0 || n > o->slots || n > MOE_MAX_TOPK) return MOE_ERR_INVALID_ARG;
   for (int i = 0; i < n; ++i) {
     if (sel[i] < 0 || sel[i] >= o->E) return MOE_ERR_INVALID_ARG;
     for (int j = 0; j < i; ++j)
       if (sel[j] == sel[i]) return MOE_ERR_INVALID_ARG;
   }
-  cudaStream_t cs = (cudaStream_t)compute_stream;
   std::vector<int>& rec = o->recency[layer];
   std::vector<int>& slot_of = o->slot_of[layer];
-  bool waited = false, any = false;
+  pl.n = n, pl.n_miss = 0;
   for (int i = 0; i < n; ++i) {
     const int e = sel[i];
+    pl.e[i] = e;
     if (slot_of[e] >= 0) {
       o->hits++;
       for (size_t p = 0; p < rec.size(); ++p)
@@ -264,6 +352,7 @@ static int ensure_impl(moe_offload* o, int32_t layer, const int32_t* sel, int32_
           break;
         }
       rec.push_back(e);
+      pl.slot[i] = slot_of[e], pl.miss[i] = false;
       continue;
     }
     int victim = -1;
@@ -274,40 +363,61 @@ static int ensure_impl(moe_offload* o, int32_t layer, const int32_t* sel, int32_
       if (!selected) victim = rec[p], vp = p;
     }
     if (victim < 0) return MOE_ERR_STATE;
-    if (!waited) {  // work already queued on the compute stream may still read the victim's slot
-      if (by_layer_event && o->layer_done_set[layer]) {
-        // the stacked steps record when a layer's kernels are done: only those read this layer's slots, so the
-        // copy need not wait for the other layers' kernels queued since
-        MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->layer_done[layer], 0));
-      } else {
-        MOE_CUDA_TRY(cudaEventRecord(o->ev_compute, cs));
-        MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->ev_compute, 0));
-      }
-      waited = true;
-    }
     const int slot = slot_of[victim];
     slot_of[victim] = -1;
     rec.erase(rec.begin() + vp);
     slot_of[e] = slot;
     rec.push_back(e);
-    unsigned char* dst = o->device_slots + ((size_t)layer * o->slots + slot) * o->slot_bytes;
-    const unsigned char* src = (const unsigned char*)o->host_experts[(size_t)layer * o->E + e];
+    pl.slot[i] = slot, pl.miss[i] = true, pl.n_miss++;
+    o->fetches++;
+    o->bytes += o->slot_bytes;
+  }
+  return MOE_OK;
+}
+
+// Work already queued on the compute stream may still read the victims' slots: the copy stream waits for it.
+// by_layer_event: the caller is a stacked step, which records layer_done[layer] after the layer's kernels -- only
+// those read this layer's slots, so the copies need not wait for the other layers' kernels queued since.
+static int copies_wait_for_readers(moe_offload* o, int32_t layer, cudaStream_t cs, bool by_layer_event) {
+  if (by_layer_event && o->layer_done_set[layer]) {
+    MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->layer_done[layer], 0));
+  } else {
+    MOE_CUDA_TRY(cudaEventRecord(o->ev_compute, cs));
+    MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->ev_compute, 0));
+  }
+  return MOE_OK;
+}
+
+// The layer's device table, rewritten in copy-stream order from a by-value copy of the host's bookkeeping.
+static int queue_table_update(moe_offload* o, int32_t layer) {
+  SlotTable tab{};
+  for (int x = 0; x < o->E; ++x) tab.slot[x] = o->slot_of[layer][x];
+  slot_table_kernel<<<1, MOE_MAX_EXPERTS, 0, o->copy_stream>>>(o->d_tables + (size_t)layer * o->E, o->E, tab);
+  MOE_CUDA_TRY(cudaGetLastError());
+  return MOE_OK;
+}
+
+static int ensure_impl(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, void* compute_stream,
+                       bool by_layer_event, LayerPlan* plan_out = nullptr) {
+  LayerPlan pl;
+  int rc = plan_layer(o, layer, sel, n, pl);
+  if (rc != MOE_OK) return rc;
+  if (plan_out) *plan_out = pl;
+  if (pl.n_miss == 0) return MOE_OK;
+  cudaStream_t cs = (cudaStream_t)compute_stream;
+  if ((rc = copies_wait_for_readers(o, layer, cs, by_layer_event)) != MOE_OK) return rc;
+  for (int i = 0; i < n; ++i) {
+    if (!pl.miss[i]) continue;
+    unsigned char* dst = o->device_slots + ((size_t)layer * o->slots + pl.slot[i]) * o->slot_bytes;
+    const unsigned char* src = (const unsigned char*)o->host_experts[(size_t)layer * o->E + pl.e[i]];
     for (size_t off = 0; off < o->slot_bytes; off += kCopyChunk) {
       const size_t nb = o->slot_bytes - off < kCopyChunk ? o->slot_bytes - off : kCopyChunk;
       MOE_CUDA_TRY(cudaMemcpyAsync(dst + off, src + off, nb, cudaMemcpyHostToDevice, o->copy_stream));
     }
-    o->fetches++;
-    o->bytes += o->slot_bytes;
-    any = true;
   }
-  if (any) {
-    SlotTable tab{};
-    for (int x = 0; x < o->E; ++x) tab.slot[x] = slot_of[x];
-    slot_table_kernel<<<1, MOE_MAX_EXPERTS, 0, o->copy_stream>>>(o->d_tables + (size_t)layer * o->E, o->E, tab);
-    MOE_CUDA_TRY(cudaGetLastError());
-    MOE_CUDA_TRY(cudaEventRecord(o->ev_copy, o->copy_stream));
-    MOE_CUDA_TRY(cudaStreamWaitEvent(cs, o->ev_copy, 0));
-  }
+  if ((rc = queue_table_update(o, layer)) != MOE_OK) return rc;
+  MOE_CUDA_TRY(cudaEventRecord(o->ev_copy, o->copy_stream));
+  MOE_CUDA_TRY(cudaStreamWaitEvent(cs, o->ev_copy, 0));
   return MOE_OK;
 }
 
@@ -336,48 +446,117 @@ int moe_offload_stats(moe_offload* o, uint64_t* fetches, uint64_t* bytes, uint64
   return MOE_OK;
 }
 
-int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* routers, float* h, int32_t* trace_host,
-                          void* ws, size_t ws_bytes, void* stream) {
-  if (!o || !ctx || !routers || !h || !ws) return MOE_ERR_INVALID_ARG;
+static int check_stack_args(moe_offload* o, moe_ctx* ctx, size_t ws_bytes) {
   const moe_config& c = ctx->cfg;
   if (c.wd_rank != 0 || c.d_model != o->cfg.d_model || c.d_ff != o->cfg.d_ff || c.n_experts != o->E ||
       c.top_k != o->cfg.top_k)
     return MOE_ERR_INVALID_ARG;
+  if (c.d_model > kRouteThreads * kRouteFeat || c.d_model > kDenseStreamMaxD) return MOE_ERR_UNSUPPORTED;
+  if (ws_bytes < ws_layout(c, 1).total) return MOE_ERR_WORKSPACE;
+  if ((size_t)c.d_ff * c.top_k * 2 < (size_t)c.d_model * 4) return MOE_ERR_UNSUPPORTED;  // u lives in the hidden region
+  return MOE_OK;
+}
+
+int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* routers, float* h, int32_t* trace_host,
+                          void* ws, size_t ws_bytes, void* stream) {
+  if (!o || !ctx || !routers || !h || !ws) return MOE_ERR_INVALID_ARG;
+  int rc = check_stack_args(o, ctx, ws_bytes);
+  if (rc != MOE_OK) return rc;
+  const moe_config& c = ctx->cfg;
   const WsLayout L = ws_layout(c, 1);
-  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
-  if ((size_t)c.d_ff * c.top_k * 2 < (size_t)c.d_model * 4) return MOE_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)stream;
   char* wsb = (char*)ws;
   int32_t* idx = (int32_t*)(wsb + L.topk_idx);
   float* wt = (float*)(wsb + L.topk_w);
-  void* u = wsb + L.hidden;               // the normalised input of the layer (x dtype; the region is >= 4*d bytes)
-  void* y = wsb + L.out_slots;            // the layer's output (x dtype)
+  void* u = wsb + L.hidden;  // the normalised input of the layer (x dtype)
   const int d = c.d_model, k = c.top_k;
   const int xbf = c.x_dtype == MOE_BF16;
+  const size_t row_bytes = (size_t)3 * d * 2;
+  using clk = std::chrono::steady_clock;
   for (int l = 0; l < o->n_layers; ++l) {
-    rms_glue_kernel<<<1, 256, 0, s>>>(h, d, u, xbf);
+    // (1) u = h / rms(h), router, selection -> device buffers and the host's mapped words
+    const int32_t seq = ++o->route_seq;
+    rms_route_kernel<<<1, kRouteThreads, 0, s>>>(h, d, o->E, k, c.renorm, (const uint16_t*)routers[l].w_router,
+                                                 routers[l].b_router, u, xbf, idx, wt, o->h_route_dev, seq);
     MOE_CUDA_TRY(cudaGetLastError());
     ctx->launches++;
-    int rc = launch_route(ctx, u, 1, &routers[l], idx, wt, nullptr, s);
-    if (rc != MOE_OK) return rc;
-    // the host issues the copies, so it has to see the selection
-    MOE_CUDA_TRY(cudaMemcpyAsync(o->h_route, idx, sizeof(int32_t) * k, cudaMemcpyDeviceToHost, s));
-    MOE_CUDA_TRY(cudaStreamSynchronize(s));
-    for (int j = 0; j < k; ++j) {
-      if (trace_host) trace_host[(size_t)l * k + j] = o->h_route[j];
+    // (2) the host must see the selection before it can queue the copies: it polls the sequence word (bounded)
+    const clk::time_point t0 = clk::now();
+    volatile int32_t* hr = o->h_route;
+    for (unsigned spin = 0; hr[k] != seq; ++spin) {
+      if ((spin & 1023u) == 1023u) {
+        if (cudaStreamQuery(s) != cudaErrorNotReady && hr[k] != seq) {  // the stream drained (or failed) without the word
+          (void)cudaGetLastError();
+          return MOE_ERR_STATE;
+        }
+        if (std::chrono::duration<double>(clk::now() - t0).count() > 10.0) return MOE_ERR_TIMEOUT;
+      }
     }
-    rc = ensure_impl(o, l, o->h_route, k, stream, true);
-    if (rc != MOE_OK) return rc;
+    std::atomic_thread_fence(std::memory_order_acquire);
+    int32_t sel[MOE_MAX_TOPK];
+    for (int j = 0; j < k; ++j) {
+      sel[j] = hr[j];
+      if (trace_host) trace_host[(size_t)l * k + j] = sel[j];
+    }
+    const clk::time_point t1 = clk::now();
+    o->t_poll += std::chrono::duration<double>(t1 - t0).count();
+    o->polls++;
+    // (3) bookkeeping; the copies of the misses go out first, chunk by chunk, each chunk with its own event
+    LayerPlan pl;
+    if ((rc = plan_layer(o, l, sel, k, pl)) != MOE_OK) return rc;
+    unsigned hit_mask = 0;
+    int last_miss = -1;
+    for (int j = 0; j < k; ++j) {
+      if (pl.miss[j])
+        last_miss = j;
+      else
+        hit_mask |= 1u << j;
+    }
+    if (pl.n_miss) {
+      if ((rc = copies_wait_for_readers(o, l, s, true)) != MOE_OK) return rc;
+      int m = 0;
+      for (int j = 0; j < k; ++j) {
+        if (!pl.miss[j]) continue;
+        unsigned char* dst = o->device_slots + ((size_t)l * o->slots + pl.slot[j]) * o->slot_bytes;
+        const unsigned char* src = (const unsigned char*)o->host_experts[(size_t)l * o->E + pl.e[j]];
+        for (int cch = 0; cch < o->n_chunks; ++cch) {
+          const int r0 = o->chunk_row[cch], r1 = o->chunk_row[cch + 1];
+          MOE_CUDA_TRY(cudaMemcpyAsync(dst + (size_t)r0 * row_bytes, src + (size_t)r0 * row_bytes, (size_t)(r1 - r0) * row_bytes,
+                                       cudaMemcpyHostToDevice, o->copy_stream));
+          MOE_CUDA_TRY(cudaEventRecord(o->chunk_ev[(size_t)m * o->n_chunks + cch], o->copy_stream));
+        }
+        ++m;
+      }
+      if ((rc = queue_table_update(o, l)) != MOE_OK) return rc;
+    }
+    // (4) the resident selected experts run while the missing ones are on their way; a missing expert is
+    // consumed chunk by chunk, each launch waiting only for its own chunk's copy.  Every launch adds into the
+    // same fixed-point accumulators; the last one converts them and adds the layer's output to h.
     moe_weights w = routers[l];
     w.gud = o->device_slots + (size_t)l * o->slots * o->slot_bytes;
-    w.expert_slot = o->d_tables + (size_t)l * o->E;
-    rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, y, nullptr, s);
-    if (rc != MOE_OK) return rc;
+    w.expert_slot = nullptr;
+    DenseExtra ex{};
+    for (int j = 0; j < MOE_MAX_TOPK; ++j) ex.slot_of_entry[j] = j < k ? pl.slot[j] : -1;
+    ex.resid = h;
+    if (hit_mask) {
+      ex.sel_mask = hit_mask, ex.unit_lo = 0, ex.unit_cnt = 0, ex.finalize = pl.n_miss == 0;
+      if ((rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, nullptr, nullptr, s, &ex)) != MOE_OK) return rc;
+    }
+    int m = 0;
+    for (int j = 0; j < k; ++j) {
+      if (!pl.miss[j]) continue;
+      for (int cch = 0; cch < o->n_chunks; ++cch) {
+        const int r0 = o->chunk_row[cch], r1 = o->chunk_row[cch + 1];
+        MOE_CUDA_TRY(cudaStreamWaitEvent(s, o->chunk_ev[(size_t)m * o->n_chunks + cch], 0));
+        ex.sel_mask = 1u << j, ex.unit_lo = r0, ex.unit_cnt = r1 - r0;
+        ex.finalize = (j == last_miss && cch == o->n_chunks - 1) ? 1 : 0;
+        if ((rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, nullptr, nullptr, s, &ex)) != MOE_OK) return rc;
+      }
+      ++m;
+    }
     MOE_CUDA_TRY(cudaEventRecord(o->layer_done[l], s));
     o->layer_done_set[l] = 1;
-    residual_kernel<<<(d + 255) / 256, 256, 0, s>>>(h, y, d, xbf);
-    MOE_CUDA_TRY(cudaGetLastError());
-    ctx->launches++;
+    o->t_issue += std::chrono::duration<double>(clk::now() - t1).count();
   }
   return MOE_OK;
 }
@@ -385,49 +564,38 @@ int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* route
 int moe_stack_decode_step_trace(moe_offload* o, moe_ctx* ctx, const moe_weights* routers, float* h,
                                 const int32_t* sel_host, void* ws, size_t ws_bytes, void* stream) {
   if (!o || !ctx || !routers || !h || !ws || !sel_host) return MOE_ERR_INVALID_ARG;
+  int rc = check_stack_args(o, ctx, ws_bytes);
+  if (rc != MOE_OK) return rc;
   const moe_config& c = ctx->cfg;
-  if (c.wd_rank != 0 || c.d_model != o->cfg.d_model || c.d_ff != o->cfg.d_ff || c.n_experts != o->E ||
-      c.top_k != o->cfg.top_k)
-    return MOE_ERR_INVALID_ARG;
-  const WsLayout L = ws_layout(c, 1);
-  if (ws_bytes < L.total) return MOE_ERR_WORKSPACE;
-  if ((size_t)c.d_ff * c.top_k * 2 < (size_t)c.d_model * 4 || (size_t)c.d_model * 2 < (size_t)c.n_experts * 4)
-    return MOE_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)stream;
-  char* wsb = (char*)ws;
-  int32_t* idx = (int32_t*)(wsb + L.topk_idx);
-  float* wt = (float*)(wsb + L.topk_w);
-  void* u = wsb + L.hidden;
-  void* y = wsb + L.out_slots;
-  float* probs = (float*)(wsb + L.xperm);  // [E] fp32; the region holds d bf16 values
-  const int d = c.d_model, k = c.top_k;
-  const int xbf = c.x_dtype == MOE_BF16;
+  const int k = c.top_k;
   for (int l = 0; l < o->n_layers; ++l) {
-    ForcedSel f{};
-    for (int j = 0; j < k; ++j) f.e[j] = sel_host[(size_t)l * k + j];
-    // the copies of this layer's misses are queued before its kernels: they run on the copy stream while the
+    // the copies of this layer's misses are queued before its kernel: they run on the copy stream while the
     // compute stream is still busy with the layers before
-    int rc = ensure_impl(o, l, f.e, k, stream, true);
+    LayerPlan pl;
+    rc = ensure_impl(o, l, sel_host + (size_t)l * k, k, stream, true, &pl);
     if (rc != MOE_OK) return rc;
-    rms_glue_kernel<<<1, 256, 0, s>>>(h, d, u, xbf);
-    MOE_CUDA_TRY(cudaGetLastError());
-    rc = launch_route(ctx, u, 1, &routers[l], idx, wt, probs, s);
-    if (rc != MOE_OK) return rc;
-    forced_routing_kernel<<<1, 32, 0, s>>>(probs, k, c.renorm, f, idx, wt);
-    MOE_CUDA_TRY(cudaGetLastError());
+    // the whole layer is one launch: u = h / rms(h), the router's probabilities of the prescribed experts, the
+    // experts, h += y
     moe_weights w = routers[l];
     w.gud = o->device_slots + (size_t)l * o->slots * o->slot_bytes;
-    w.expert_slot = o->d_tables + (size_t)l * o->E;
-    rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, y, nullptr, s);
+    w.expert_slot = nullptr;
+    DenseExtra ex{};
+    for (int j = 0; j < MOE_MAX_TOPK; ++j) ex.slot_of_entry[j] = j < k ? pl.slot[j] : -1, ex.forced[j] = j < k ? pl.e[j] : 0;
+    ex.finalize = 1, ex.resid = h, ex.h_in = h, ex.use_forced = 1;
+    rc = launch_dense_stream(ctx, 0, h, 1, &w, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, s, &ex);
     if (rc != MOE_OK) return rc;
     MOE_CUDA_TRY(cudaEventRecord(o->layer_done[l], s));
     o->layer_done_set[l] = 1;
-    residual_kernel<<<(d + 255) / 256, 256, 0, s>>>(h, y, d, xbf);
-    MOE_CUDA_TRY(cudaGetLastError());
-    ctx->launches += 3;
   }
-  // the per-layer staging of the slot tables is reused by the next step
-  MOE_CUDA_TRY(cudaStreamSynchronize(s));
+  return MOE_OK;
+}
+
+int moe_offload_host_times(moe_offload* o, double* poll_s, double* issue_s, uint64_t* polls) {
+  if (!o) return MOE_ERR_INVALID_ARG;
+  if (poll_s) *poll_s = o->t_poll;
+  if (issue_s) *issue_s = o->t_issue;
+  if (polls) *polls = o->polls;
   return MOE_OK;
 }
 

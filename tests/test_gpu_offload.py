@@ -54,12 +54,11 @@ def test_stacked_decode_with_offload_matches_checker(slots):
                 U.assert_valid_tied_selection(sel[l], ora["logits"][0], sh.top_k, (step, l))
                 ora = O.layer_forward(xin, host[l]["w_router"], host[l]["b_router"], ex, sh.top_k,
                                       forced_topk=np.int32([sel[l]]))
-            y_b = torch.from_numpy(ora["y"][0].astype(np.float32)).to(torch.bfloat16).double().numpy()
-            hh = hh + y_b
+            hh = hh + ora["y"][0]                       # h += y in fp32 on the device, y not rounded in between
             traces[l].append(sel[l])
         got = h.cpu().numpy().astype(np.float64)
-        # rounding of u and y to bf16 happens at the same places on both sides; what is left is fp32 vs fp64
-        # arithmetic inside the layers, amplified by at most n_layers
+        # u is rounded to bf16 at the same place on both sides; what is left is fp32 vs fp64 arithmetic inside the
+        # layers, amplified by at most n_layers
         U.assert_close_rms(got, hh, tol=U.Y_TOL, what=f"h after step {step}")
     # bookkeeping: fetches, bytes, hits and the final residents, exactly, on the GPU's own routing
     st = stack.stats()
@@ -100,7 +99,7 @@ def test_stacked_decode_with_prescribed_expert_sets(p_stay):
             ex = {k: v for k, v in host[l].items() if k not in ("w_router", "b_router")}
             ora = O.layer_forward(W.to_host_bits(u_b[None]), host[l]["w_router"], host[l]["b_router"], ex, sh.top_k,
                                   forced_topk=np.int32([sel[l]]))
-            hh = hh + torch.from_numpy(ora["y"][0].astype(np.float32)).to(torch.bfloat16).double().numpy()
+            hh = hh + ora["y"][0]
         U.assert_close_rms(h.cpu().numpy().astype(np.float64), hh, tol=U.Y_TOL, what=f"h after step {step}")
     st = stack.stats()
     tot = {"n_fetch": 0, "bytes": 0, "hits": 0}
@@ -207,3 +206,48 @@ def test_expert_replacements_reads_rows_as_sets():
             if 0 <= e < 4:
                 A[0, t, e] = 1
     assert int(out.item()) == X.hard_replacements(A)[1]
+
+
+def test_stacked_decode_with_offload_at_the_phone_shape():
+    """The offload configuration at its real widths (d 2048, f 5632, E 16, 4 resident experts per layer), a few
+    layers and steps: one expert is 69 MB, so a fetch is nine chunks, every chunk its own launch over a range of
+    hidden units that waits for that chunk's copy, all launches of a layer adding into the same accumulators.
+    Outputs against the fp64 chain, fetches / bytes / hits / residents against the cache simulation."""
+    sh = W.PHONE_OFFLOAD
+    n_layers, steps, slots = 4, 6, 4
+    stack, host = make_stack(sh, n_layers, slots)
+    torch.cuda.empty_cache()
+    traces = [[] for _ in range(n_layers)]
+    for step in range(steps):
+        h0 = W.make_x(sh.with_(x_dtype="f32"), 1, device="cuda", step=step)[0].contiguous()
+        h = h0.clone()
+        sel = stack.step(h)
+        torch.cuda.synchronize()
+        assert stack.check() == 0
+        hh = h0.cpu().numpy().astype(np.float64)
+        for l in range(n_layers):
+            u = O.rms_glue(hh[None])[0]
+            u_b = torch.from_numpy(u.astype(np.float32)).to(torch.bfloat16)
+            xin = W.to_host_bits(u_b[None])
+            ex = {k: v for k, v in host[l].items() if k not in ("w_router", "b_router")}
+            R = O.router_logits(xin, host[l]["w_router"], host[l]["b_router"])
+            tie = O.near_tie_tokens(R, sh.top_k, U.TIE_GAP)[0]
+            if tie:
+                U.assert_valid_tied_selection(sel[l], R[0], sh.top_k, (step, l))
+            ora = O.layer_forward(xin, host[l]["w_router"], host[l]["b_router"], ex, sh.top_k,
+                                  forced_topk=np.int32([sel[l]]) if tie else None)
+            if not tie:
+                assert sel[l] == ora["topk_idx"][0].tolist(), (step, l, sel[l], ora["topk_idx"][0])
+            hh = hh + ora["y"][0]
+            traces[l].append(sel[l])
+        U.assert_close_rms(h.cpu().numpy().astype(np.float64), hh, tol=U.Y_TOL, what=f"h after step {step}")
+    st = stack.stats()
+    tot = {"n_fetch": 0, "bytes": 0, "hits": 0}
+    for l in range(n_layers):
+        sim = F.lru_cache_sim(traces[l], sh.n_experts, slots, stack.slot_bytes)
+        for k in tot:
+            tot[k] += sim[k]
+        assert stack.resident(l) == sim["slots"][-1]
+    assert (st["fetches"], st["bytes"], st["hits"]) == (tot["n_fetch"], tot["bytes"], tot["hits"])
+    assert st["fetches"] > 0 and st["hits"] > 0          # both kinds of layer were met
+    stack.close()
