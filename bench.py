@@ -5,9 +5,11 @@
 
 One step = one forward pass of the whole layer (router, top-k gating, grouping, expert FFN,
 gate-weighted combine) over one batch of seeded synthetic input.  The default workload is the
-wearables-scale layer at batch-1 decode; steps walk a ring of distinct layers whose touched
-weights exceed the L2 several times over, so every step reads its experts from HBM.
-Prints ONE JSON line (see the keys below).  N > 1: independent replicas, one per GPU, no collective.
+phone-scale layer at batch-1 decode (the largest single-GPU decode configuration); steps walk a ring of
+distinct layers whose touched weights exceed the L2 several times over, so every step reads its experts
+from HBM.  Prints ONE JSON line; unless --no-others is given it also times the other configurations
+(decode and prefill, dense and weight-decomposed experts, a shortened offload stack) and reports them
+under "others", each with its roofline.  N > 1: independent replicas, one per GPU, no collective.
 """
 from __future__ import annotations
 
@@ -41,7 +43,11 @@ WORKLOADS = {
     "phone-wd1024-prefill-T2048": (W.PHONE_WD1024, 2048, "prefill"),
     "tiny-T16": (W.TINY, 16, "decode"),
 }
-DEFAULT = "wearable-decode-T1"
+DEFAULT = "phone-decode-T1"
+# timed after the main workload and reported under "others" (the offload stack, shortened, is added to them)
+OTHERS = ["wearable-decode-T1", "wearable-decode-T8", "wearable-prefill-T512", "phone-prefill-T2048",
+          "phone-wd128-decode-T1", "phone-wd1024-decode-T1", "phone-wd128-prefill-T2048", "phone-wd1024-prefill-T2048"]
+NOMINAL = {"hbm_gbs": 8000.0, "tflops": 2250.0}   # the target's denominators: about 8 TB/s, dense bf16 2.25 PFLOP/s
 
 # Shape sweep (--sweep): batch-1 decode over the paper's ablation grid -- active experts k in {1, 2, 4, 8} at E = 8,
 # total experts E in {2, 4, 8, 16} at k = 2 (Fig. 7: time grows with k, not with E) -- and the paper's own layer
@@ -150,7 +156,7 @@ def run_ring(ring, steps, start=0):
         r["layer"].forward(r["x"], y=r["y"], topk_idx=r["idx"], topk_w=r["w"])
 
 
-def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use_graph=True):
+def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use_graph=True, min_ms=1500.0):
     shape, T, kind = WORKLOADS[name]
     pk = peaks()
     ring = build_ring(shape, T, device, 4 * L2_BYTES, ring_override)
@@ -184,8 +190,10 @@ def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use
             sys.stderr.write(f"[bench] CUDA graph capture unavailable ({e}); timing plain launches\n")
             torch.cuda.synchronize()
             graph = None
-    trips = max(1, steps // n) if graph is not None else None
-    steps_eff = trips * n if graph is not None else steps
+    # whole trips around the ring, rounded up; the same trips are repeated until the timed region is long enough
+    # for the clock samplers (this one and any outside) to see the load
+    trips = -(-steps // n)
+    steps_trip = trips * n
 
     def timed_once():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -197,7 +205,7 @@ def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use
             for _ in range(trips):
                 graph.replay()
         else:
-            run_ring(ring, steps_eff)
+            run_ring(ring, steps_trip)
         e1.record()
         torch.cuda.synchronize()
         if world > 1:
@@ -208,14 +216,13 @@ def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use
     if sampler:
         sampler.start()
     ms = timed_once()
-    # keep the GPU busy long enough for at least a few clock samples
-    extra_ms, reps = 0.0, 0
-    while sampler and (extra_ms + ms) < 400.0 and reps < 50:
-        extra_ms += timed_once()
-        reps += 1
+    reps = 1
+    if world == 1:          # replicas keep to the steps asked for: every rank must run the same number of regions
+        while ms < min_ms and reps < 100000:
+            ms += timed_once()
+            reps += 1
     clocks = sampler.stop() if sampler else None
-    if reps:
-        ms = (ms + extra_ms) / (reps + 1)
+    steps_eff = steps_trip * reps
     for r in ring:
         assert r["layer"].check() == 0, "a kernel flagged an error during the timed region"
 
@@ -232,21 +239,46 @@ def _launches(r):
     return B.moe_launch_count(r["layer"].ctx)
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
-# under profiles/ (same workload, ring of fewer layers).  An entry is dropped when its kernel changes.
-NCU_TRAFFIC_BYTES = {
-    "wearable-decode-T1": 34_782_976,                    # dense_stream_kernel, one launch per step
-    "wearable-decode-T8": 121_376_256 + 3_742_720,       # dense_stream_kernel, launch with 7 active experts
-    "phone-prefill-T2048": 473_914_112 + 40_779_008,     # grouped_gemm_kernel, the first (larger) GEMM of the layer
-    "phone-decode-T1": 138_686_976 + 3_785_472,          # dense_stream_kernel
-    "phone-wd128-decode-T1": 11_899_904,                 # wd_decode_kernel
-    "phone-wd1024-decode-T1": 94_490_624 + 3_387_392,    # stream_ffn_kernel
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel come from the ncu summaries under
+# profiles/ (same workload, ring of fewer layers).  A summary carries the lines
+#     traffic_bytes_per_launch: <bytes>
+#     kernel_source: <file under csrc/> sha256 <hex>
+# and its figure is used only while that source file is unchanged: once the kernel has been edited the counters
+# no longer describe it and "traffic" is null until the capture is retaken.
+PROFILE_OF = {
+    "wearable-decode-T1": "dense_stream_kernel_wearable_decode_T1.md",
+    "wearable-decode-T8": "dense_stream_kernel_wearable_decode_T8.md",
+    "phone-decode-T1": "dense_stream_kernel_phone_decode_T1.md",
+    "phone-prefill-T2048": "grouped_gemm_kernel_phone_prefill_T2048.md",
+    "phone-wd128-decode-T1": "wd_decode_kernel_phone_wd128_decode_T1.md",
+    "phone-wd1024-decode-T1": "stream_ffn_kernel_phone_wd1024_decode_T1.md",
 }
+
+
+def ncu_traffic(name):
+    import hashlib
+    import re
+    fn = PROFILE_OF.get(name)
+    path = os.path.join(ROOT, "profiles", fn) if fn else None
+    if not path or not os.path.exists(path):
+        return None
+    text = open(path).read()
+    m = re.search(r"^traffic_bytes_per_launch:\s*(\d+)", text, re.M)
+    k = re.search(r"^kernel_source:\s*(\S+)\s+sha256\s+([0-9a-f]{64})", text, re.M)
+    if not m or not k:
+        return None
+    src = os.path.join(ROOT, "paper_2503_00245_b200", "csrc", k.group(1))
+    if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != k.group(2):
+        return None
+    return int(m.group(1))
 
 
 def roofline(res):
     r = _roofline(res)
-    r["traffic"] = NCU_TRAFFIC_BYTES.get(res.get("name"))
+    r["traffic"] = ncu_traffic(res.get("name"))
+    nominal = NOMINAL["hbm_gbs"] if r["bound"] == "hbm" else NOMINAL["tflops"]
+    r["peak_nominal"] = nominal
+    r["frac_nominal"] = round(r["achieved"] / nominal, 4)
     return r
 
 
@@ -347,7 +379,7 @@ def cpu_baseline(name, budget_s=12.0):
             "sample": f"{n} forward passes of layer 0 of the ring ({el:.1f} s of CPU time), numpy fp64"}
 
 
-def run_offload_stack(a, device):
+def run_offload_stack(a, device, emit=True):
     """Stacked decode with host-resident experts: n_layers phone-scale layers (E = 16, top-2), `slots` experts
     per layer resident in HBM, the rest in pinned host memory, Zipf(1.2)-skewed routing; one step = one token
     through all layers.  Reports us/token and the host-link traffic against the measured pinned H2D rate."""
@@ -386,6 +418,7 @@ def run_offload_stack(a, device):
         stack.step(hs[steps + s].clone())
     torch.cuda.synchronize()
     st0 = stack.stats()
+    ht0 = B.moe_offload_host_times(stack.off)
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
     trace = []
@@ -409,6 +442,14 @@ def run_offload_stack(a, device):
     B.moe_expert_replacements(tr, n_layers, steps, sh.top_k, sh.n_experts, hsum)
     torch.cuda.synchronize()
     exrep = (int(hsum.item()) // 2) / (n_layers * sh.top_k * max(1, steps - 1))
+    # expert balance per layer (Section 3.3): mean over the layers of the deviation from the uniform share, percent
+    cnt = torch.zeros((n_layers, sh.n_experts), dtype=torch.int64, device=device)
+    dlt = torch.zeros(n_layers + 1, dtype=torch.float64, device=device)
+    bad = torch.zeros(1, dtype=torch.int64, device=device)
+    B.moe_delta_uniform(tr, n_layers, steps, sh.top_k, sh.n_experts, cnt, dlt, bad)
+    torch.cuda.synchronize()
+    delta_uniform = float(dlt[n_layers].item())
+    ht1 = B.moe_offload_host_times(stack.off)
     us_tok = ms * 1e3 / steps
     bytes_tok = nbytes / steps
     t_link = bytes_tok / (h2d_gbs * 1e9) * 1e6
@@ -419,7 +460,8 @@ def run_offload_stack(a, device):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/activations, f32 accumulate",
         "data": "synthetic",
         "config": {"workload": "phone-offload-stack", "shape": W.describe(sh), "layers": n_layers,
-                   "resident_slots_per_layer": slots, "T": 1, "launch_mode": "stream (host sync per layer)",
+                   "resident_slots_per_layer": slots, "T": 1, "decode_steps": steps,
+                   "launch_mode": "stream (the host polls a mapped routing word per layer)",
                    "l2": "inputs larger than L2: 24 distinct layers per token"},
         "roofline": {"bound": "host_link", "achieved": round(bytes_tok / (us_tok * 1e-6) / 1e9, 2),
                      "peak": round(h2d_gbs, 2), "unit": "GB/s",
@@ -428,16 +470,26 @@ def run_offload_stack(a, device):
                      "note": "frac = (fetch bytes / measured H2D rate) / time per token"},
         "offload": {"fetch_bytes_per_token": int(bytes_tok), "fetches_per_token": round(fetches / steps, 3),
                     "hit_rate": round(hits / lookups, 4), "exrep": round(exrep, 4),
+                    "delta_uniform_pct": round(delta_uniform, 3),
                     "no_miss_floor_us": round(t_hbm, 1), "host_link_floor_us": round(t_link, 1),
-                    "host_wall_us_per_token": round(wall * 1e6 / steps, 1)},
+                    "host_wall_us_per_token": round(wall * 1e6 / steps, 1),
+                    # where a token's time goes besides the link: the host waiting for routing words (the device is
+                    # then computing the layer's last chunk and the next layer's norm + router) and queueing work
+                    "host_poll_us_per_token": round((ht1["poll_s"] - ht0["poll_s"]) * 1e6 / steps, 1),
+                    "host_issue_us_per_token": round((ht1["issue_s"] - ht0["issue_s"]) * 1e6 / steps, 1),
+                    "link_idle_us_per_token": round(us_tok - t_link, 1)},
         "e2e": {"value": round(wall * 1e6 / steps, 2), "unit": "us/token", "h2d_bytes_per_step": int(bytes_tok),
                 "d2h_bytes_per_step": n_layers * sh.top_k * 4},
         "gpu_launches": int(B.moe_launch_count(stack.ctx)),
         "clocks": clocks,
     }
-    print(json.dumps(line))
     stack.close()
-    return 0
+    del stack
+    torch.cuda.empty_cache()
+    if emit:
+        print(json.dumps(line))
+        return 0
+    return line
 
 
 def run_offload_eq8(a, device):
@@ -560,7 +612,9 @@ def main():
     ap.add_argument("--layers", type=int, default=24, help="phone-offload-stack: stacked layers")
     ap.add_argument("--slots", type=int, default=4, help="phone-offload-stack: resident experts per layer")
     ap.add_argument("--decode-steps", type=int, default=256, help="phone-offload-stack: tokens")
-    ap.add_argument("--all", action="store_true", help="also time the other workloads (reported under 'others')")
+    ap.add_argument("--all", action="store_true", help="(default behaviour now; kept for old command lines)")
+    ap.add_argument("--no-others", action="store_true", help="time the main workload only")
+    ap.add_argument("--others-offload-steps", type=int, default=32, help="tokens of the shortened offload stack in 'others'")
     ap.add_argument("--sweep", action="store_true", help="also time the shape sweep (reported under 'sweep')")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -611,23 +665,33 @@ def main():
     _, e2e_val, _, _ = metric_of(res, max_over_ranks(e2e_ms, world, device), world)
 
     others = []
-    if a.all and rank == 0 and world == 1:
+    if not a.no_others and rank == 0 and world == 1 and a.workload == DEFAULT:
         res.pop("ring", None)
         torch.cuda.empty_cache()
-        for name in WORKLOADS:
-            if name == a.workload or name in SWEEP:
-                continue
+        for name in OTHERS:
             try:
-                r = time_workload(name, a.steps, a.warmup, device, rank, 1)
+                r = time_workload(name, min(a.steps, 1024), a.warmup, device, rank, 1, min_ms=400.0)
             except Exception as e:  # noqa: BLE001
                 others.append({"workload": name, "error": str(e)[:200]})
                 continue
             m, v, u, _ = metric_of(r, r["ms_per_step"])
-            others.append({"workload": name, "metric": m, "value": round(v, 3), "unit": u,
+            others.append({"workload": name, "metric": m, "value": round(v, 3), "unit": u, "steps": r["steps"],
                            "ms_per_step": round(r["ms_per_step"], 5), "launch_mode": r["launch_mode"],
-                           "active_experts_per_step": r["active_experts_per_step"], "roofline": roofline(r)})
+                           "launches_per_step": r["launches_per_step"],
+                           "active_experts_per_step": r["active_experts_per_step"], "roofline": roofline(r),
+                           "clocks": r["clocks"]})
             del r
             torch.cuda.empty_cache()
+        try:
+            saved = a.decode_steps
+            a.decode_steps = a.others_offload_steps
+            o = run_offload_stack(a, device, emit=False)
+            a.decode_steps = saved
+            others.append({"workload": "phone-offload-stack", "metric": o["metric"], "value": o["value"], "unit": o["unit"],
+                           "steps": o["steps"], "ms_per_step": o["ms_per_step"], "config": o["config"],
+                           "roofline": o["roofline"], "offload": o["offload"], "clocks": o["clocks"]})
+        except Exception as e:  # noqa: BLE001
+            others.append({"workload": "phone-offload-stack", "error": str(e)[:200]})
 
     sweep = []
     if a.sweep and rank == 0 and world == 1:

@@ -172,3 +172,39 @@ def test_argument_errors_are_reported_not_run():
     assert e.value.status == 2                      # streaming path is limited to 16 tokens
     B.moe_layer_forward(lay.ctx, t["x"], 0, lay.weights, y, ws=lay.ws)   # T = 0: no-op
     assert lay.check() == 0
+
+
+def _decode_us(sh, reps=200):
+    """Median-free, simple timing of batch-1 decode over a ring of distinct layers (weights beyond L2 are not
+    needed for a comparison between shapes: every shape is timed the same way)."""
+    lays = [U.build(sh, 1, layer=l)[0] for l in range(6)]
+    x = W.make_x(sh, 1, device="cuda")
+    ys = [torch.empty_like(x) for _ in lays]
+    for _ in range(3):
+        for lay, y in zip(lays, ys):
+            lay.forward(x, y=y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        for lay, y in zip(lays, ys):
+            lay.forward(x, y=y)
+    e1.record()
+    torch.cuda.synchronize()
+    for lay in lays:
+        assert lay.check() == 0
+        lay.close()
+    return e0.elapsed_time(e1) * 1e3 / (reps * len(lays))
+
+
+def test_decode_time_follows_active_not_total_experts():
+    """The paper's ablation (Section 3.4.4, Fig. 7): generation speed falls with the number of ACTIVE experts and
+    does not depend on the TOTAL number, because only the selected experts' weights are touched.  Wearable widths,
+    batch-1 decode; generous bounds (a launch has a fixed cost besides the weight stream)."""
+    base = W.WEARABLE
+    t_k1 = _decode_us(base.with_(top_k=1))
+    t_k8 = _decode_us(base.with_(top_k=8))
+    t_e2 = _decode_us(base.with_(n_experts=2))
+    t_e16 = _decode_us(base.with_(n_experts=16))
+    assert t_k8 > 2.0 * t_k1, (t_k1, t_k8)
+    assert abs(t_e16 - t_e2) < 0.2 * max(t_e16, t_e2), (t_e2, t_e16)
