@@ -287,7 +287,7 @@ def _decode_kernel_name(shape, T):
     if not shape.wd_rank:
         return "dense_stream_kernel"
     wd_bytes = shape.top_k * W.expert_bytes(shape)
-    return "wd_decode_kernel" if (T == 1 and wd_bytes <= 32 * 1024 * 1024) else "stream_ffn_kernel"
+    return ("wd_decode_kernel" if wd_bytes <= 32 * 1024 * 1024 else "wd_stream_kernel") if T == 1 else "stream_ffn_kernel"
 
 
 def _roofline(res):
