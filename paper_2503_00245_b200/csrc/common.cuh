@@ -36,9 +36,7 @@ struct DeviceState {
   unsigned long long done_total;
   // weight-decomposed decode kernel: arrivals at its meetings between the products, counted the same way
   unsigned long long phase_total;
-  // grouped GEMM: next tile to hand out.  The GEMMs of a layer alternate between the two words; each one clears
-  // the other word for its successor, and the row gather clears word 0 for the first.
-  unsigned int tile_ctr[2];
+  unsigned int pad_tail[2];
   unsigned int pad3[26];
 };
 
@@ -82,7 +80,7 @@ constexpr int kKSplitMax = 4;          // planes the tensor path may ask for ...
 constexpr int kKSplitMaxSlots = 2048;  // ... when there are at most this many (token, choice) slots
 int launch_combine(moe_ctx* ctx, const float* out_slots, const float* wt, const int32_t* inv, int T, void* y,
                    int planes, cudaStream_t s);
-int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_slots, void* xperm, cudaStream_t s);  // also clears tile_ctr[0]
+int launch_gather_rows(moe_ctx* ctx, const void* x, const int32_t* perm, int n_slots, void* xperm, cudaStream_t s);
 
 // Streaming (decode) path.  mode 0: whole layer from topk (writes y); mode 1: FFN per slot from
 // expert_offsets/perm (writes out_slots).

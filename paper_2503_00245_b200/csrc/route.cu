@@ -332,7 +332,6 @@ __global__ void gather_rows_kernel(const XT* __restrict__ x, const int32_t* __re
   const long long total = (long long)n_slots * chunks;
   pdl_launch_dependents();
   pdl_wait();
-  if (blockIdx.x == 0 && threadIdx.x == 0) st->tile_ctr[0] = 0u;  // the first GEMM after this kernel draws its tiles from it
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const int s = (int)(i / chunks), c = (int)(i % chunks);
