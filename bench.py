@@ -251,7 +251,7 @@ PROFILE_OF = {
     "phone-decode-T1": "dense_stream_kernel_phone_decode_T1.md",
     "phone-prefill-T2048": "grouped_gemm_kernel_phone_prefill_T2048.md",
     "phone-wd128-decode-T1": "wd_decode_kernel_phone_wd128_decode_T1.md",
-    "phone-wd1024-decode-T1": "stream_ffn_kernel_phone_wd1024_decode_T1.md",
+    "phone-wd1024-decode-T1": "wd_stream_kernel_phone_wd1024_decode_T1.md",
 }
 
 
@@ -620,6 +620,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ring", type=int, default=0, help="override the number of distinct layers in the ring")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of a CUDA graph")
+    ap.add_argument("--min-ms", type=float, default=1500.0,
+                    help="repeat the timed steps until the region is at least this long (0: exactly --steps, for profiling)")
     a = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -658,7 +660,7 @@ def main():
         return run_offload_stack(a, device) if rank == 0 else 0
     if a.workload == "phone-offload-eq8":
         return run_offload_eq8(a, device) if rank == 0 else 0
-    res = time_workload(a.workload, a.steps, a.warmup, device, rank, world, a.ring, not a.no_graph)
+    res = time_workload(a.workload, a.steps, a.warmup, device, rank, world, a.ring, not a.no_graph, a.min_ms)
     ms_per_step = max_over_ranks(res["ms_total"], world, device) / res["steps"]
     metric, value, unit, hib = metric_of(res, ms_per_step, world)
     e2e_ms, h2d, d2h = e2e_measure(res, a.steps)
