@@ -379,7 +379,7 @@ def cpu_baseline(name, budget_s=12.0):
             "sample": f"{n} forward passes of layer 0 of the ring ({el:.1f} s of CPU time), numpy fp64"}
 
 
-def run_offload_stack(a, device, emit=True):
+def run_offload_stack(a, device, emit=True, fp8=False):
     """Stacked decode with host-resident experts: n_layers phone-scale layers (E = 16, top-2), `slots` experts
     per layer resident in HBM, the rest in pinned host memory, Zipf(1.2)-skewed routing; one step = one token
     through all layers.  Reports us/token and the host-link traffic against the measured pinned H2D rate."""
@@ -399,7 +399,7 @@ def run_offload_stack(a, device, emit=True):
         for lay in layers:
             yield lay
             lay["gud"] = None          # the device copy is no longer needed once it is in pinned memory
-    stack = P.OffloadedStack(sh.d_model, sh.d_ff, sh.n_experts, sh.top_k, slots, gen())
+    stack = P.OffloadedStack(sh.d_model, sh.d_ff, sh.n_experts, sh.top_k, slots, gen(), fp8=fp8)
     torch.cuda.empty_cache()
     # pinned host->device bandwidth of this machine (the roofline of a miss)
     probe_dst = torch.empty(stack.slot_bytes, dtype=torch.uint8, device=device)
@@ -459,7 +459,8 @@ def run_offload_stack(a, device, emit=True):
         "n_gpus": 1, "steps": steps, "warmup": 3, "ms_per_step": round(ms / steps, 4), "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/activations, f32 accumulate",
         "data": "synthetic",
-        "config": {"workload": "phone-offload-stack", "shape": W.describe(sh), "layers": n_layers,
+        "config": {"workload": "phone-offload-stack-fp8" if fp8 else "phone-offload-stack", "shape": W.describe(sh),
+                   "host_copies": "FP8 E4M3 codes + fp32 row scales" if fp8 else "bf16", "layers": n_layers,
                    "resident_slots_per_layer": slots, "T": 1, "decode_steps": steps,
                    "launch_mode": "stream (the host polls a mapped routing word per layer)",
                    "l2": "inputs larger than L2: 24 distinct layers per token"},
@@ -614,6 +615,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=256, help="phone-offload-stack: tokens")
     ap.add_argument("--all", action="store_true", help="(default behaviour now; kept for old command lines)")
     ap.add_argument("--no-others", action="store_true", help="time the main workload only")
+    ap.add_argument("--fp8-host", action="store_true", help="phone-offload-stack: host copies as FP8 codes + row scales")
     ap.add_argument("--others-offload-steps", type=int, default=32, help="tokens of the shortened offload stack in 'others'")
     ap.add_argument("--sweep", action="store_true", help="also time the shape sweep (reported under 'sweep')")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -657,7 +659,7 @@ def main():
         torch.distributed.barrier()
 
     if a.workload == "phone-offload-stack":
-        return run_offload_stack(a, device) if rank == 0 else 0
+        return run_offload_stack(a, device, fp8=a.fp8_host) if rank == 0 else 0
     if a.workload == "phone-offload-eq8":
         return run_offload_eq8(a, device) if rank == 0 else 0
     res = time_workload(a.workload, a.steps, a.warmup, device, rank, world, a.ring, not a.no_graph, a.min_ms)
@@ -684,16 +686,18 @@ def main():
                            "clocks": r["clocks"]})
             del r
             torch.cuda.empty_cache()
-        try:
-            saved = a.decode_steps
-            a.decode_steps = a.others_offload_steps
-            o = run_offload_stack(a, device, emit=False)
-            a.decode_steps = saved
-            others.append({"workload": "phone-offload-stack", "metric": o["metric"], "value": o["value"], "unit": o["unit"],
-                           "steps": o["steps"], "ms_per_step": o["ms_per_step"], "config": o["config"],
-                           "roofline": o["roofline"], "offload": o["offload"], "clocks": o["clocks"]})
-        except Exception as e:  # noqa: BLE001
-            others.append({"workload": "phone-offload-stack", "error": str(e)[:200]})
+        saved = a.decode_steps
+        a.decode_steps = a.others_offload_steps
+        for fp8 in (False, True):
+            name = "phone-offload-stack-fp8" if fp8 else "phone-offload-stack"
+            try:
+                o = run_offload_stack(a, device, emit=False, fp8=fp8)
+                others.append({"workload": name, "metric": o["metric"], "value": o["value"], "unit": o["unit"],
+                               "steps": o["steps"], "ms_per_step": o["ms_per_step"], "config": o["config"],
+                               "roofline": o["roofline"], "offload": o["offload"], "clocks": o["clocks"]})
+            except Exception as e:  # noqa: BLE001
+                others.append({"workload": name, "error": str(e)[:200]})
+        a.decode_steps = saved
 
     sweep = []
     if a.sweep and rank == 0 and world == 1:

@@ -137,6 +137,13 @@ int moe_pack_wd(int32_t d_model, int32_t d_ff, int32_t rank, int32_t n_experts, 
                 const void* uL, const void* uR, const void* dL, const void* dR, void* wd_a_out, void* wd_b_out,
                 void* wd_c_out, void* wd_d_out, void* stream);
 
+/* ---- 8-bit storage of packed rows (for the host link) -----------------------------
+ * rows x n bf16 values (dev, n a multiple of 8) -> FP8 E4M3 codes (dev [rows][n] bytes) and one fp32 scale per
+ * row: scale = max|w| / 448 (1 for an all-zero row), code = e4m3(w / scale) with round-to-nearest-even and
+ * saturation, all in fp32.  moe_fp8_dequantize_rows: w' = bf16(value(code) * scale).                      */
+int moe_fp8_quantize_rows(const void* w, int64_t rows, int32_t n, void* codes, float* scales, void* stream);
+int moe_fp8_dequantize_rows(const void* codes, const float* scales, int64_t rows, int32_t n, void* w, void* stream);
+
 /* ---- the layer, step by step ---------------------------------------------------- */
 
 /* Router logits, softmax over experts (Eq. 2), top-k (Eq. 3), gate weights.
@@ -209,6 +216,16 @@ int moe_layer_forward_static(const moe_config* cfg, const void* x, int32_t T, co
  * in stream order, and the call returns without waiting for the copies.           */
 int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_per_layer,
                        const void* const* host_experts, void* device_slots, size_t slot_bytes, moe_offload** out);
+/* The same with the host copies in 8-bit form (bit-width reduction for the host link; the paper names it only as
+ * related work, Section 2.3 / Section 5): host_blobs[layer*E + e] -> pinned memory holding the expert's packed
+ * rows as FP8 E4M3 codes, [f][3][d] bytes, followed by one fp32 scale per row, [f][3] (moe_fp8_quantize_rows makes
+ * both from the packed bf16 rows).  A fetch moves d_ff * (3 d + 12) bytes instead of 6 d d_ff, lands in a staging
+ * area the object owns and is widened into the bf16 slot by a kernel ordered behind the copy (on the compute stream
+ * in the stacked steps, so that the copy stream only ever copies); the layer kernels read
+ * bf16 slots as before, so the layer computes with w' = bf16(value(code) * scale) in place of w.
+ * slot_bytes stays the bf16 size of a slot (6 d d_ff).                                                       */
+int moe_offload_create_fp8(const moe_config* cfg, int32_t n_layers, int32_t slots_per_layer,
+                           const void* const* host_blobs, void* device_slots, size_t slot_bytes, moe_offload** out);
 int moe_offload_destroy(moe_offload* off);
 int moe_offload_ensure(moe_offload* off, int32_t layer, const int32_t* topk_idx_host, int32_t n,
                        void* compute_stream);

@@ -61,6 +61,10 @@ _SIGS = {
     "moe_layer_forward_static": (C.c_int, [C.POINTER(moe_config), _P, C.c_int32, C.POINTER(moe_weights), _P, _P, _P, _P]),
     "moe_offload_create": (C.c_int, [C.POINTER(moe_config), C.c_int32, C.c_int32, C.POINTER(_P), _P, C.c_size_t,
                                      C.POINTER(_P)]),
+    "moe_offload_create_fp8": (C.c_int, [C.POINTER(moe_config), C.c_int32, C.c_int32, C.POINTER(_P), _P, C.c_size_t,
+                                         C.POINTER(_P)]),
+    "moe_fp8_quantize_rows": (C.c_int, [_P, C.c_int64, C.c_int32, _P, _P, _P]),
+    "moe_fp8_dequantize_rows": (C.c_int, [_P, _P, C.c_int64, C.c_int32, _P, _P]),
     "moe_offload_destroy": (C.c_int, [_P]),
     "moe_offload_ensure": (C.c_int, [_P, C.c_int32, C.POINTER(C.c_int32), C.c_int32, _P]),
     "moe_offload_slot_table": (C.c_int, [_P, C.c_int32, C.POINTER(_P)]),
@@ -201,12 +205,15 @@ def moe_layer_forward_static(cfg: moe_config, x, T, w: moe_weights, y, topk_idx=
                                            _ptr(topk_w), _stream(stream))
 
 
-def moe_offload_create(cfg: moe_config, n_layers, slots_per_layer, host_expert_ptrs, device_slots, slot_bytes) -> int:
-    """host_expert_ptrs: sequence of n_layers*E host addresses (pinned memory the caller keeps alive)."""
+def moe_offload_create(cfg: moe_config, n_layers, slots_per_layer, host_expert_ptrs, device_slots, slot_bytes,
+                       fp8=False) -> int:
+    """host_expert_ptrs: sequence of n_layers*E host addresses (pinned memory the caller keeps alive); with fp8 they
+    point to FP8 blobs (codes, then row scales) and moe_offload_create_fp8 is called."""
     arr = (C.c_void_p * len(host_expert_ptrs))(*host_expert_ptrs)
     h = _P()
-    _ok(_lib().moe_offload_create(C.byref(cfg), n_layers, slots_per_layer, arr, _ptr(device_slots), slot_bytes,
-                                  C.byref(h)), "moe_offload_create")
+    fn = _lib().moe_offload_create_fp8 if fp8 else _lib().moe_offload_create
+    _ok(fn(C.byref(cfg), n_layers, slots_per_layer, arr, _ptr(device_slots), slot_bytes, C.byref(h)),
+        "moe_offload_create_fp8" if fp8 else "moe_offload_create")
     _KEEP[h.value] = arr
     return h.value
 
@@ -272,3 +279,12 @@ def moe_offload_host_times(off: int):
     a, b, n = C.c_double(), C.c_double(), C.c_uint64()
     _ok(_lib().moe_offload_host_times(off, C.byref(a), C.byref(b), C.byref(n)), "moe_offload_host_times")
     return {"poll_s": a.value, "issue_s": b.value, "polls": n.value}
+
+
+def moe_fp8_quantize_rows(w, rows, n, codes, scales, stream=None):
+    _ok(_lib().moe_fp8_quantize_rows(_ptr(w), rows, n, _ptr(codes), _ptr(scales), _stream(stream)), "moe_fp8_quantize_rows")
+
+
+def moe_fp8_dequantize_rows(codes, scales, rows, n, w, stream=None):
+    _ok(_lib().moe_fp8_dequantize_rows(_ptr(codes), _ptr(scales), rows, n, _ptr(w), _stream(stream)),
+        "moe_fp8_dequantize_rows")

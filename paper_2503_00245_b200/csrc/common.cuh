@@ -109,6 +109,8 @@ bool dense_stream_fuses_route(const moe_config& c, int T);  // mode 0 computes t
 int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_weights* w, int32_t* topk_idx,
                         float* topk_w, const int32_t* offsets, const int32_t* perm, void* y, float* out_slots,
                         cudaStream_t s, const DenseExtra* ex = nullptr);
+// FP8 E4M3 codes with one fp32 scale per row of n values -> bf16 (csrc/fp8_store.cu).
+int launch_fp8_dequant(const void* codes, const float* scales, long long rows, int n, void* w, cudaStream_t s);
 // Tensor-core (prefill) path: out_slots from x gathered by perm.
 int launch_tensor_ffn(moe_ctx* ctx, const void* x, int T, const moe_weights* w, const int32_t* offsets,
                       const int32_t* perm, char* ws, const WsLayout& L, float* out_slots, int* out_planes,

@@ -37,6 +37,12 @@ struct moe_offload {
   std::vector<int> chunk_row;               // a missing expert is copied (and computed) in runs of hidden units
   int n_chunks;                             // [chunk_row[c], chunk_row[c+1]): halves of what is left, so that few copies are
                                             // issued and the compute that trails the last one is short
+  int fp8;                                  // the host copies are FP8 codes + row scales (half the link bytes)
+  size_t blob_bytes;                        // bytes of one expert on the host: slot_bytes, or codes + scales
+  unsigned char* staging;                   // device, fp8 only: [2][top_k] blobs as they arrive, before widening into the slot
+                                            // (two sets, by layer parity: a layer's copies may run while the layer before is widened)
+  cudaEvent_t staging_free[2];              // recorded on the compute stream after a set's last widening kernel
+  char staging_used[2];
   uint64_t fetches, bytes, hits;
   // what the routed step spent where, summed over its calls (host wall time, seconds)
   double t_poll, t_issue;
@@ -46,8 +52,7 @@ struct moe_offload {
 namespace cosmoe {
 namespace {
 
-constexpr size_t kCopyChunk = 8u << 20;  // moe_offload_ensure issues its host->device copies in chunks of this size
-constexpr size_t kLastChunk = 4u << 20;  // stacked steps: a miss is copied in halves of the rest, down to about this size
+constexpr size_t kLastChunk = 4u << 20;  // a miss is copied in halves of what is left, down to about this size
 
 // A layer's expert -> slot table, passed BY VALUE: every queued update carries its own copy, so a later call
 // for the same layer cannot change what an earlier, still pending update writes.
@@ -223,8 +228,62 @@ using namespace cosmoe;
 
 extern "C" {
 
+static int offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_per_layer,
+                          const void* const* host_experts, void* device_slots, size_t slot_bytes, int fp8, moe_offload** out);
+
 int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_per_layer,
                        const void* const* host_experts, void* device_slots, size_t slot_bytes, moe_offload** out) {
+  return offload_create(cfg, n_layers, slots_per_layer, host_experts, device_slots, slot_bytes, 0, out);
+}
+
+int moe_offload_create_fp8(const moe_config* cfg, int32_t n_layers, int32_t slots_per_layer,
+                           const void* const* host_blobs, void* device_slots, size_t slot_bytes, moe_offload** out) {
+  return offload_create(cfg, n_layers, slots_per_layer, host_blobs, device_slots, slot_bytes, 1, out);
+}
+
+// Copy of one expert's rows [r0, r1) from the host, on the copy stream.  bf16 host copies go straight into the
+// device slot.  FP8 blobs (codes [f][3][d], then scales [f][3]) land in the staging area of miss number `m` of the
+// layer (set layer & 1); widen_rows turns them into the slot's bf16 rows on whatever stream the caller orders
+// behind the copy -- the compute stream in the stacked steps, so that the copy stream only ever copies.
+static unsigned char* staging_of(moe_offload* o, int layer, int m) {
+  return o->staging + ((size_t)(layer & 1) * o->cfg.top_k + m) * o->blob_bytes;
+}
+static int queue_rows(moe_offload* o, int layer, int e, int slot, int m, int r0, int r1) {
+  const size_t d = (size_t)o->cfg.d_model, f = (size_t)o->cfg.d_ff;
+  const unsigned char* src = (const unsigned char*)o->host_experts[(size_t)layer * o->E + e];
+  if (!o->fp8) {
+    unsigned char* dst = o->device_slots + ((size_t)layer * o->slots + slot) * o->slot_bytes;
+    const size_t row_bytes = 3 * d * 2;
+    MOE_CUDA_TRY(cudaMemcpyAsync(dst + (size_t)r0 * row_bytes, src + (size_t)r0 * row_bytes, (size_t)(r1 - r0) * row_bytes,
+                                 cudaMemcpyHostToDevice, o->copy_stream));
+    return MOE_OK;
+  }
+  unsigned char* stg = staging_of(o, layer, m);
+  const size_t codes_bytes = f * 3 * d;
+  if (r0 == 0)  // the scales of the whole expert go first (12 f bytes)
+    MOE_CUDA_TRY(cudaMemcpyAsync(stg + codes_bytes, src + codes_bytes, f * 3 * sizeof(float), cudaMemcpyHostToDevice, o->copy_stream));
+  MOE_CUDA_TRY(cudaMemcpyAsync(stg + (size_t)r0 * 3 * d, src + (size_t)r0 * 3 * d, (size_t)(r1 - r0) * 3 * d, cudaMemcpyHostToDevice,
+                               o->copy_stream));
+  return MOE_OK;
+}
+static int widen_rows(moe_offload* o, int layer, int slot, int m, int r0, int r1, cudaStream_t s) {
+  if (!o->fp8) return MOE_OK;
+  const size_t d = (size_t)o->cfg.d_model, f = (size_t)o->cfg.d_ff;
+  unsigned char* stg = staging_of(o, layer, m);
+  unsigned char* dst = o->device_slots + ((size_t)layer * o->slots + slot) * o->slot_bytes;
+  return launch_fp8_dequant(stg + (size_t)r0 * 3 * d, reinterpret_cast<const float*>(stg + f * 3 * d) + (size_t)r0 * 3,
+                            (long long)(r1 - r0) * 3, (int)d, dst + (size_t)r0 * 3 * d * 2, s);
+}
+// The staging set of `layer` is free again once the widening kernels queued on `s` so far have run.
+static int staging_release(moe_offload* o, int layer, cudaStream_t s) {
+  if (!o->fp8) return MOE_OK;
+  MOE_CUDA_TRY(cudaEventRecord(o->staging_free[layer & 1], s));
+  o->staging_used[layer & 1] = 1;
+  return MOE_OK;
+}
+
+static int offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_per_layer,
+                          const void* const* host_experts, void* device_slots, size_t slot_bytes, int fp8, moe_offload** out) {
   if (!out) return MOE_ERR_INVALID_ARG;
   *out = nullptr;
   int rc = validate_config(cfg);
@@ -241,6 +300,9 @@ int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_pe
   o->device_slots = (unsigned char*)device_slots;
   o->slot_bytes = slot_bytes;
   o->fetches = o->bytes = o->hits = 0;
+  o->fp8 = fp8, o->staging = nullptr;
+  o->staging_free[0] = o->staging_free[1] = nullptr, o->staging_used[0] = o->staging_used[1] = 0;
+  o->blob_bytes = fp8 ? (size_t)cfg->d_ff * 3 * cfg->d_model + (size_t)cfg->d_ff * 3 * sizeof(float) : slot_bytes;
   o->copy_stream = nullptr, o->ev_compute = nullptr, o->ev_copy = nullptr;
   o->d_tables = nullptr, o->h_tables = nullptr, o->h_route = nullptr, o->h_route_dev = nullptr;
   o->route_seq = 0, o->t_poll = o->t_issue = 0.0, o->polls = 0;
@@ -271,6 +333,8 @@ int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_pe
     for (size_t i = 0; i < o->chunk_ev.size() && e == cudaSuccess; ++i)
       e = cudaEventCreateWithFlags(&o->chunk_ev[i], cudaEventDisableTiming);
   }
+  if (e == cudaSuccess && fp8) e = cudaMalloc((void**)&o->staging, (size_t)2 * cfg->top_k * o->blob_bytes);
+  for (int i = 0; i < 2 && e == cudaSuccess && fp8; ++i) e = cudaEventCreateWithFlags(&o->staging_free[i], cudaEventDisableTiming);
   if (e == cudaSuccess) {
     o->layer_done.assign(n_layers, nullptr);
     o->layer_done_set.assign(n_layers, 0);
@@ -284,8 +348,8 @@ int moe_offload_create(const moe_config* cfg, int32_t n_layers, int32_t slots_pe
       for (int s = 0; s < o->slots && e == cudaSuccess; ++s) {  // slot s starts with expert s, expert 0 oldest
         o->recency[l].push_back(s);
         o->slot_of[l][s] = s;
-        e = cudaMemcpyAsync(o->device_slots + ((size_t)l * o->slots + s) * slot_bytes,
-                            host_experts[(size_t)l * o->E + s], slot_bytes, cudaMemcpyHostToDevice, o->copy_stream);
+        if (queue_rows(o, l, s, s, 0, 0, cfg->d_ff) != MOE_OK || widen_rows(o, l, s, 0, 0, cfg->d_ff, o->copy_stream) != MOE_OK)
+          e = cudaErrorUnknown;
       }
       for (int x = 0; x < o->E; ++x) o->h_tables[(size_t)l * o->E + x] = o->slot_of[l][x];
     }
@@ -314,6 +378,9 @@ int moe_offload_destroy(moe_offload* o) {
     if (ev) cudaEventDestroy(ev);
   for (cudaEvent_t ev : o->chunk_ev)
     if (ev) cudaEventDestroy(ev);
+  if (o->staging) cudaFree(o->staging);
+  for (int i = 0; i < 2; ++i)
+    if (o->staging_free[i]) cudaEventDestroy(o->staging_free[i]);
   if (o->d_tables) cudaFree(o->d_tables);
   if (o->h_tables) cudaFreeHost(o->h_tables);
   if (o->h_route) cudaFreeHost(o->h_route);
@@ -370,7 +437,7 @@ static int plan_layer(moe_offload* o, int32_t layer, const int32_t* sel, int32_t
     rec.push_back(e);
     pl.slot[i] = slot, pl.miss[i] = true, pl.n_miss++;
     o->fetches++;
-    o->bytes += o->slot_bytes;
+    o->bytes += o->blob_bytes;
   }
   return MOE_OK;
 }
@@ -379,6 +446,8 @@ static int plan_layer(moe_offload* o, int32_t layer, const int32_t* sel, int32_t
 // by_layer_event: the caller is a stacked step, which records layer_done[layer] after the layer's kernels -- only
 // those read this layer's slots, so the copies need not wait for the other layers' kernels queued since.
 static int copies_wait_for_readers(moe_offload* o, int32_t layer, cudaStream_t cs, bool by_layer_event) {
+  if (o->fp8 && o->staging_used[layer & 1])  // the staging set's last contents have been widened
+    MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->staging_free[layer & 1], 0));
   if (by_layer_event && o->layer_done_set[layer]) {
     MOE_CUDA_TRY(cudaStreamWaitEvent(o->copy_stream, o->layer_done[layer], 0));
   } else {
@@ -406,19 +475,21 @@ static int ensure_impl(moe_offload* o, int32_t layer, const int32_t* sel, int32_
   if (pl.n_miss == 0) return MOE_OK;
   cudaStream_t cs = (cudaStream_t)compute_stream;
   if ((rc = copies_wait_for_readers(o, layer, cs, by_layer_event)) != MOE_OK) return rc;
-  for (int i = 0; i < n; ++i) {
+  for (int i = 0, m = 0; i < n; ++i) {
     if (!pl.miss[i]) continue;
-    unsigned char* dst = o->device_slots + ((size_t)layer * o->slots + pl.slot[i]) * o->slot_bytes;
-    const unsigned char* src = (const unsigned char*)o->host_experts[(size_t)layer * o->E + pl.e[i]];
-    for (size_t off = 0; off < o->slot_bytes; off += kCopyChunk) {
-      const size_t nb = o->slot_bytes - off < kCopyChunk ? o->slot_bytes - off : kCopyChunk;
-      MOE_CUDA_TRY(cudaMemcpyAsync(dst + off, src + off, nb, cudaMemcpyHostToDevice, o->copy_stream));
-    }
+    for (int cch = 0; cch < o->n_chunks; ++cch)
+      if ((rc = queue_rows(o, layer, pl.e[i], pl.slot[i], m, o->chunk_row[cch], o->chunk_row[cch + 1])) != MOE_OK) return rc;
+    ++m;
   }
   if ((rc = queue_table_update(o, layer)) != MOE_OK) return rc;
   MOE_CUDA_TRY(cudaEventRecord(o->ev_copy, o->copy_stream));
   MOE_CUDA_TRY(cudaStreamWaitEvent(cs, o->ev_copy, 0));
-  return MOE_OK;
+  for (int i = 0, m = 0; i < n; ++i) {  // 8-bit host copies: widened on the compute stream, behind the copies
+    if (!pl.miss[i]) continue;
+    if ((rc = widen_rows(o, layer, pl.slot[i], m, 0, o->cfg.d_ff, cs)) != MOE_OK) return rc;
+    ++m;
+  }
+  return staging_release(o, layer, cs);
 }
 
 int moe_offload_ensure(moe_offload* o, int32_t layer, const int32_t* sel, int32_t n, void* compute_stream) {
@@ -471,7 +542,6 @@ int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* route
   void* u = wsb + L.hidden;  // the normalised input of the layer (x dtype)
   const int d = c.d_model, k = c.top_k;
   const int xbf = c.x_dtype == MOE_BF16;
-  const size_t row_bytes = (size_t)3 * d * 2;
   using clk = std::chrono::steady_clock;
   for (int l = 0; l < o->n_layers; ++l) {
     // (1) u = h / rms(h), router, selection -> device buffers and the host's mapped words
@@ -517,12 +587,8 @@ int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* route
       int m = 0;
       for (int j = 0; j < k; ++j) {
         if (!pl.miss[j]) continue;
-        unsigned char* dst = o->device_slots + ((size_t)l * o->slots + pl.slot[j]) * o->slot_bytes;
-        const unsigned char* src = (const unsigned char*)o->host_experts[(size_t)l * o->E + pl.e[j]];
         for (int cch = 0; cch < o->n_chunks; ++cch) {
-          const int r0 = o->chunk_row[cch], r1 = o->chunk_row[cch + 1];
-          MOE_CUDA_TRY(cudaMemcpyAsync(dst + (size_t)r0 * row_bytes, src + (size_t)r0 * row_bytes, (size_t)(r1 - r0) * row_bytes,
-                                       cudaMemcpyHostToDevice, o->copy_stream));
+          if ((rc = queue_rows(o, l, pl.e[j], pl.slot[j], m, o->chunk_row[cch], o->chunk_row[cch + 1])) != MOE_OK) return rc;
           MOE_CUDA_TRY(cudaEventRecord(o->chunk_ev[(size_t)m * o->n_chunks + cch], o->copy_stream));
         }
         ++m;
@@ -548,12 +614,14 @@ int moe_stack_decode_step(moe_offload* o, moe_ctx* ctx, const moe_weights* route
       for (int cch = 0; cch < o->n_chunks; ++cch) {
         const int r0 = o->chunk_row[cch], r1 = o->chunk_row[cch + 1];
         MOE_CUDA_TRY(cudaStreamWaitEvent(s, o->chunk_ev[(size_t)m * o->n_chunks + cch], 0));
+        if ((rc = widen_rows(o, l, pl.slot[j], m, r0, r1, s)) != MOE_OK) return rc;
         ex.sel_mask = 1u << j, ex.unit_lo = r0, ex.unit_cnt = r1 - r0;
         ex.finalize = (j == last_miss && cch == o->n_chunks - 1) ? 1 : 0;
         if ((rc = launch_dense_stream(ctx, 2, u, 1, &w, idx, wt, nullptr, nullptr, nullptr, nullptr, s, &ex)) != MOE_OK) return rc;
       }
       ++m;
     }
+    if (pl.n_miss && (rc = staging_release(o, l, s)) != MOE_OK) return rc;
     MOE_CUDA_TRY(cudaEventRecord(o->layer_done[l], s));
     o->layer_done_set[l] = 1;
     o->t_issue += std::chrono::duration<double>(clk::now() - t1).count();

@@ -123,25 +123,39 @@ class OffloadedStack:
     """n_layers stacked MoE layers whose experts live in pinned host memory (packed gud layout); the device
     keeps `slots` experts per layer.  Owns the pinned master copy, the device slots, a ctx and its workspace."""
 
-    def __init__(self, d_model, d_ff, n_experts, top_k, slots, layers, x_dtype=torch.bfloat16, device="cuda"):
-        """layers: iterable of dicts with w_router, b_router and gud [E,f,3,d] (device tensors, consumed one by one)."""
+    def __init__(self, d_model, d_ff, n_experts, top_k, slots, layers, x_dtype=torch.bfloat16, device="cuda", fp8=False):
+        """layers: iterable of dicts with w_router, b_router and gud [E,f,3,d] (device tensors, consumed one by one).
+        fp8: keep the host copies as FP8 codes + row scales (half the bytes per fetch)."""
         import ctypes
+        self.fp8 = fp8
         self.d, self.f, self.E, self.k, self.slots = d_model, d_ff, n_experts, top_k, slots
         self.cfg = B.make_config(d_model, d_ff, n_experts, top_k, 0,
                                  B.MOE_F32 if x_dtype == torch.float32 else B.MOE_BF16, 1, B.MOE_PATH_STREAM)
         self.slot_bytes = d_ff * 3 * d_model * 2
         self.host, self.routers_t = [], []
         ptrs = []
+        self.blob_bytes = d_ff * 3 * d_model + d_ff * 3 * 4 if fp8 else self.slot_bytes
         for lay in layers:
-            hg = torch.empty(lay["gud"].shape, dtype=torch.bfloat16, pin_memory=True)
-            hg.copy_(lay["gud"])
+            if fp8:
+                gud = lay["gud"]
+                rows = n_experts * d_ff * 3
+                codes = torch.empty((n_experts, d_ff * 3 * d_model), dtype=torch.uint8, device=gud.device)
+                scales = torch.empty((n_experts, d_ff * 3), dtype=torch.float32, device=gud.device)
+                B.moe_fp8_quantize_rows(gud, rows, d_model, codes, scales)
+                hg = torch.empty((n_experts, self.blob_bytes), dtype=torch.uint8, pin_memory=True)
+                hg[:, :d_ff * 3 * d_model].copy_(codes)
+                hg[:, d_ff * 3 * d_model:].copy_(scales.view(torch.uint8).reshape(n_experts, -1))
+                del codes, scales
+            else:
+                hg = torch.empty(lay["gud"].shape, dtype=torch.bfloat16, pin_memory=True)
+                hg.copy_(lay["gud"])
             self.host.append(hg)
             self.routers_t.append((lay["w_router"], lay["b_router"]))
-            ptrs += [hg.data_ptr() + e * self.slot_bytes for e in range(n_experts)]
+            ptrs += [hg.data_ptr() + e * self.blob_bytes for e in range(n_experts)]
         self.n_layers = len(self.host)
         torch.cuda.synchronize()
         self.device_slots = torch.empty(self.n_layers * slots * self.slot_bytes, dtype=torch.uint8, device=device)
-        self.off = B.moe_offload_create(self.cfg, self.n_layers, slots, ptrs, self.device_slots, self.slot_bytes)
+        self.off = B.moe_offload_create(self.cfg, self.n_layers, slots, ptrs, self.device_slots, self.slot_bytes, fp8=fp8)
         self.ctx = B.moe_create(self.cfg)
         self.ws = torch.empty(B.moe_workspace_bytes(self.cfg, 1), dtype=torch.uint8, device=device)
         self.routers = (B.moe_weights * self.n_layers)()
