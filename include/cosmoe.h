@@ -173,7 +173,10 @@ int moe_combine(moe_ctx* ctx, const float* out_slots, const float* topk_w, const
                 void* stream);
 
 /* The whole layer: equals moe_route -> moe_permute -> moe_expert_ffn -> moe_combine
- * but is free to fuse.  topk_idx / topk_w (dev, may be NULL) receive the routing.   */
+ * but is free to fuse.  topk_idx / topk_w (dev, may be NULL) receive the routing.
+ * On the streaming path (T <= MOE_STREAM_MAX_TOKENS) y may also be MAPPED PINNED HOST memory (a device-accessible
+ * address): the finalising CTAs store y with ordinary stores, so a decode step then needs no device->host copy,
+ * only a wait for `stream` before the host reads y.                                  */
 int moe_layer_forward(moe_ctx* ctx, const void* x, int32_t T, const moe_weights* w, void* y, int32_t* topk_idx,
                       float* topk_w, void* ws, size_t ws_bytes, void* stream);
 

@@ -99,7 +99,8 @@ def _ptr(t) -> int | None:
         return None
     if isinstance(t, int):
         return t
-    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    # device tensors, or pinned host tensors (mapped: the device reaches them at the same address)
+    assert (t.is_cuda or t.is_pinned()) and t.is_contiguous(), "device-resident (or pinned host) contiguous tensors only"
     return t.data_ptr()
 
 

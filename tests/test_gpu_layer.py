@@ -208,3 +208,18 @@ def test_decode_time_follows_active_not_total_experts():
     t_e16 = _decode_us(base.with_(n_experts=16))
     assert t_k8 > 2.0 * t_k1, (t_k1, t_k8)
     assert abs(t_e16 - t_e2) < 0.2 * max(t_e16, t_e2), (t_e2, t_e16)
+
+
+@pytest.mark.parametrize("sh,T", [(W.WEARABLE, 1), (W.PHONE, 1), (W.TINY, 16), (W.WEARABLE, 8)])
+def test_streaming_path_writes_y_to_mapped_host_memory(sh, T):
+    """On the streaming path y may be mapped pinned host memory: the finalising CTAs store it themselves."""
+    lay, t, _ = U.build(sh, T, path=STREAM)
+    for step in range(2):
+        x = W.make_x(sh, T, device="cuda", step=step)
+        ref = lay.forward(x)
+        hy = torch.zeros((T, sh.d_model), dtype=x.dtype).pin_memory()
+        lay.forward(x, y=hy)
+        torch.cuda.synchronize()
+        assert lay.check() == 0
+        assert torch.equal(hy, ref.cpu())
+    lay.close()
