@@ -36,8 +36,10 @@ struct DeviceState {
   unsigned long long done_total;
   // weight-decomposed decode kernel: arrivals at its meetings between the products, counted the same way
   unsigned long long phase_total;
-  unsigned int pad_tail[2];
-  unsigned int pad3[26];
+  // dense streaming kernel, one token: next stage (4 hidden units) of each active expert that no CTA has taken yet;
+  // the finalisers leave zeros
+  unsigned int stage_ctr[MOE_MAX_TOPK];
+  unsigned int pad3[20];
 };
 
 }  // namespace cosmoe

@@ -67,6 +67,7 @@ struct DenseParams {
   long long fin_wait_budget;   // cycles a finalising CTA waits for the arrival counter to fill up
   int f_full;                  // hidden units per expert in memory (f may be a sub-range of them, starting at ex.unit_lo)
   int given1;                  // one token, routing taken from topk_idx / topk_w (possibly a subset of its entries)
+  int dyn;                     // one token, d > 1024: stages are handed out from per-expert counters (see consume_pass_cols)
   DenseExtra ex;
 };
 
@@ -76,6 +77,7 @@ struct Smem {
   uint64_t freeb[kMaxStages];  // all consumer warps are done with the stage
   uint64_t xfull[2];           // token rows of a pass landed in xs[0/1]
   uint64_t cbar;               // barrier over the consumer warps
+  int stage_n[kMaxStages];             // dynamic hand-out: hidden units in the stage (0 = no more stages)
   float gu[kMaxStages][kRows * 2];     // single-token passes at d > 1024: the stage's 8 dot products
   __align__(16) float red[4][2][kRows * 8][kWarps];  // multi-token passes: [stage index & 3][gate | up][unit * 8 + token][warp]
   __align__(16) uint32_t zero16[4];    // what ldmatrix reads for padding rows
@@ -100,6 +102,7 @@ struct Pass {
 struct PassIt {
   int ai, ai_hi, grp, ngrp, ra, rb;
   unsigned u0, u1;
+  int cta_j, cta_c;  // few active experts: this CTA is number cta_j of the cta_c that work for its expert (else cta_c = 0)
 };
 
 __device__ __forceinline__ void item_bounds(const Smem& sm, int f, PassIt& g) {
@@ -117,6 +120,7 @@ __device__ __forceinline__ void item_bounds(const Smem& sm, int f, PassIt& g) {
 __device__ __forceinline__ void pass_split(unsigned na, int f, PassIt& g) {
   const unsigned G = gridDim.x, b = blockIdx.x;
   g.ra = g.rb = g.grp = g.ngrp = 0;
+  g.cta_j = g.cta_c = 0;
   if (na > 0 && na <= 16u && G >= na) {
     // few active experts: every CTA works for ONE expert (a second pass costs its set-up and its output atomics
     // again); the first G % na experts get one CTA more than the others
@@ -128,6 +132,7 @@ __device__ __forceinline__ void pass_split(unsigned na, int f, PassIt& g) {
       const unsigned b2 = b - extra * (base + 1u);
       ai = extra + b2 / base, j = b2 % base, c = base;
     }
+    g.cta_j = (int)j, g.cta_c = (int)c;
     g.u0 = ai * (unsigned)f + j * (unsigned)f / c;  // j * f < 2^23
     g.u1 = ai * (unsigned)f + (j + 1u) * (unsigned)f / c;
   } else {
@@ -557,8 +562,9 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
   const bool owner = mychunk < cw1;
   const int cclamp = owner ? mychunk : cw0;
   float acc[8];
+  long long iacc[8];  // dynamic hand-out: fixed-point sums, so that the result does not depend on which CTA took which stage
 #pragma unroll
-  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f, iacc[j] = 0;
   float4 xr[kXIters][2];
 #pragma unroll
   for (int it = 0; it < kXIters; ++it) {
@@ -567,12 +573,13 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
   }
   const float wgt = sm.slot_w[slot0];
 
-  for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
-    const int nrows = min(kRows, ps.rb - row0);
+  for (int row0 = ps.ra; P.dyn || row0 < ps.rb; row0 += kRows) {
     if (!mbar_wait(&sm.full[rp.slot], rp.par)) {
       if (lane == 0) set_abort(st, sm, 0x310u);
       return false;
     }
+    const int nrows = P.dyn ? sm.stage_n[rp.slot] : min(kRows, ps.rb - row0);
+    if (nrows == 0) break;  // dynamic hand-out: the producer found no stage left
     const unsigned char* stage = ring + (size_t)rp.slot * P.stage_bytes;
     const int r = warp >> 1;
     if (r < nrows) {
@@ -618,6 +625,10 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[j] = fmaf(h, w[j], acc[j]);
     }
+    if (P.dyn) {  // a stage's sum depends on the stage alone; integer addition across stages is associative
+#pragma unroll
+      for (int j = 0; j < 8; ++j) iacc[j] += __float2ll_rn(acc[j] * kFixScale), acc[j] = 0.f;
+    }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.freeb[rp.slot]);
     rp.advance(NS);
@@ -627,7 +638,7 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
     unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) +
                               (size_t)(blockIdx.x % P.acc_copies) * P.acc_copy_stride + (size_t)rowi * d + mychunk * 8;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) atomicAdd(dst + j, (unsigned long long)__float2ll_rn(acc[j] * kFixScale));
+    for (int j = 0; j < 8; ++j) atomicAdd(dst + j, (unsigned long long)(P.dyn ? iacc[j] : __float2ll_rn(acc[j] * kFixScale)));
   }
   return true;
 }
@@ -1081,8 +1092,22 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       }
       const unsigned char* src = reinterpret_cast<const unsigned char*>(P.gud) +
                                  ((size_t)sm.act_slot[ps.ai] * P.f_full + P.ex.unit_lo + ps.ra) * row_bytes;
-      for (int row = ps.ra; row < ps.rb; row += kRows) {
-        const uint32_t bytes = (uint32_t)min(kRows, ps.rb - row) * row_bytes;
+      // Dynamic hand-out (one token, one pass per CTA): the CTAs of an expert do not stream at the same rate -- equal
+      // shares end up to 4 us apart at the phone shape -- so a CTA takes half of its equal share of the
+      // expert's stages (4 hidden units each) statically and then draws single stages from the expert's counter until
+      // none is left.  A stage with zero units tells the consumers that the pass is over.
+      const int n_st = (P.f + kRows - 1) / kRows;
+      const int dyn_s0 = P.dyn ? (int)((long long)n_st / (2 * pit.cta_c)) : 0;
+      int dyn_next = pit.cta_j * dyn_s0;
+      const int dyn_stat_end = dyn_next + dyn_s0, dyn_base = pit.cta_c * dyn_s0;
+      for (int row = ps.ra; P.dyn || row < ps.rb; row += kRows) {
+        int cur = 0;
+        if (P.dyn) {
+          cur = dyn_next < dyn_stat_end ? dyn_next++ : dyn_base + (int)atomicAdd(&st->stage_ctr[ps.ai], 1u);
+          if (cur >= n_st) cur = -1;
+        }
+        const int nrows = P.dyn ? (cur < 0 ? 0 : min(kRows, P.f - cur * kRows)) : min(kRows, ps.rb - row);
+        const uint32_t bytes = (uint32_t)nrows * row_bytes;
         if (rp.n >= NS) {
           if (!mbar_wait(&sm.freeb[rp.slot], rp.par ^ 1u)) {
             set_abort(st, sm, 0x330u);
@@ -1094,6 +1119,16 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         if (sm.abort) {
           ok = false;
           break;
+        }
+        if (P.dyn) {
+          sm.stage_n[rp.slot] = nrows;
+          if (nrows == 0) {  // no stage left: the consumers leave on this one
+            mbar_arrive(&sm.full[rp.slot]);
+            rp.advance(NS);
+            break;
+          }
+          src = reinterpret_cast<const unsigned char*>(P.gud) +
+                ((size_t)sm.act_slot[ps.ai] * P.f_full + P.ex.unit_lo + (size_t)cur * kRows) * row_bytes;
         }
         fence_proxy_async_smem();
         mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
@@ -1185,6 +1220,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   fin = consumer_sync(sm, cpar, lane) && fin;
   const int slice = sm.last;
   if (fin && slice >= 0) {
+    if (slice == 0 && tid < MOE_MAX_TOPK) st->stage_ctr[tid] = 0u;  // every CTA has arrived: nobody draws stages any more
     const int rows = P.mode == 0 ? P.T : n_pairs;
     const long long total = (long long)rows * P.d;
     const long long per = (total + K - 1) / K;
@@ -1303,6 +1339,11 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
   const int v = !P.use_mma ? (P.wpart_ok ? V_T1 : V_COLS)
                            : (c.d_model <= 1024 ? (P.x_is_bf16 ? V_MMA_BF16_S : V_MMA_F32_S)
                                                 : (P.x_is_bf16 ? V_MMA_BF16_L : V_MMA_F32_L));
+  P.dyn = (v == V_COLS && mode == 0 && T == 1 && P.ex.finalize && P.ex.unit_cnt == 0 &&
+           (P.ex.sel_mask & ((1u << c.top_k) - 1u)) == (1u << c.top_k) - 1u &&
+           G >= c.top_k && c.d_ff >= 8 * G)
+              ? 1
+              : 0;
   int rc;
   switch (v) {
     case V_T1: rc = launch_variant<V_T1>(P, G, smem, s); break;
@@ -1405,7 +1446,7 @@ extern "C" int moe_layer_forward_static(const moe_config* cfg, const void* x, in
   if (T > 1 && (!topk_idx || !topk_w)) return MOE_ERR_INVALID_ARG;
   // The array keeps what the last call left.  A call that ran to its end leaves the accumulators and the
   // arrival counter at zero, one that was cut short does not: clear the part this call uses, keep the status.
-  MOE_CUDA_TRY(cudaMemsetAsync(&st->done_total, 0, sizeof(unsigned long long), s));
+  MOE_CUDA_TRY(cudaMemsetAsync(&st->done_total, 0, offsetof(DeviceState, pad3) - offsetof(DeviceState, done_total), s));  // arrival and stage counters
   MOE_CUDA_TRY(cudaMemsetAsync(acc, 0, kStaticAccBytes, s));
   moe_ctx tmp{};  // a view, not a context: nothing here owns memory
   tmp.cfg = *cfg;
