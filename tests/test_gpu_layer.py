@@ -89,9 +89,15 @@ def test_all_tokens_to_one_expert_stream():
     assert ora["counts"].tolist() == [0, 0, 16, 0, 0, 16, 0, 0]
 
 
-def test_layer_equals_composition_of_steps():
-    sh = W.WEARABLE
-    lay, t, host = U.build(sh, 8)
+@pytest.mark.parametrize("sh,T", [
+    (W.WEARABLE, 8),                       # fused streaming kernel against the four calls (streaming FFN per slot)
+    (W.PHONE, 1),                          # one launch with dynamic stage hand-out against the four calls
+    (shape(1440, 3840), 300),              # tensor path: layer (route, permute, gather, two GEMMs, combine) against the calls
+    (W.PHONE_WD1024, 1),                   # streamed factor products in one launch against the four-phase per-slot kernel
+    (shape(256, 512, r=64, xd="f32"), 7),
+])
+def test_layer_equals_composition_of_steps(sh, T):
+    lay, t, host = U.build(sh, T)
     y = lay.forward(t["x"])
     idx, w, _ = lay.route(t["x"])
     offsets, perm, inv = lay.permute(idx)
