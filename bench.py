@@ -195,32 +195,32 @@ def time_workload(name, steps, warmup, device, rank, world, ring_override=0, use
     trips = -(-steps // n)
     steps_trip = trips * n
 
-    def timed_once():
+    def timed_region(n_trips):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
         e0.record()
         if graph is not None:
-            for _ in range(trips):
+            for _ in range(n_trips):
                 graph.replay()
         else:
-            run_ring(ring, steps_trip)
+            run_ring(ring, n_trips * n)
         e1.record()
         torch.cuda.synchronize()
         if world > 1:
             torch.distributed.barrier()
         return e0.elapsed_time(e1)
 
+    # one untimed region of the steps asked for tells how many repeats make the timed region long enough; the
+    # timed region is then ONE bracket (barrier + synchronise on both sides) around all of them
+    reps = 1
+    if world == 1 and min_ms > 0:   # replicas keep to the steps asked for: every rank runs the same region
+        reps = max(1, int(-(-min_ms // max(timed_region(trips), 1e-3))))
     sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
     if sampler:
         sampler.start()
-    ms = timed_once()
-    reps = 1
-    if world == 1:          # replicas keep to the steps asked for: every rank must run the same number of regions
-        while ms < min_ms and reps < 100000:
-            ms += timed_once()
-            reps += 1
+    ms = timed_region(trips * reps)
     clocks = sampler.stop() if sampler else None
     steps_eff = steps_trip * reps
     for r in ring:
