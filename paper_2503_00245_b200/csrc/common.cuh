@@ -252,6 +252,11 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ unsigned ld_relaxed(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -341,40 +346,65 @@ __device__ __forceinline__ float f32_unkey(unsigned k) {
 // bits than fp32 probabilities); ties go to the lower expert index.  Lane j < k writes the j-th choice.
 // (maxima go through the warp's integer reduction, one instruction instead of five shuffle rounds: this
 // routine sits on the serial path of every decode launch)
+// Registers only: lane j < k gets the j-th choice (my_idx) and its gate weight (my_w); every lane gets the set of
+// selected experts as a bit mask.  One warp-wide maximum and one ballot per choice; the exponentials are those of
+// the k selected logits only, unless the full softmax is asked for (probs_out) or the weights are not renormalised
+// (then the softmax denominator over all E logits is needed).  Renormalised weights are formed the same way in
+// either case, exp(l_j - m) / sum over the selected of exp(l_i - m) with m the largest logit, so they do not depend
+// on whether the probabilities were asked for.
+__device__ __forceinline__ void warp_route_top(float l0, float l1, int E, int k, int renorm, int lane,
+                                               float* __restrict__ probs_out, int& my_idx, float& my_w,
+                                               unsigned long long& selmask) {
+  const unsigned FULL = 0xffffffffu;
+  const bool has0 = lane < E, has1 = lane + 32 < E;
+  const bool two = E > 32;  // (uniform) a lane holds a second logit
+  unsigned key0 = has0 ? f32_key(l0) : 0u, key1 = has1 ? f32_key(l1) : 0u;  // 0: taken or absent (below every key)
+  float m = 0.f, wtot = 0.f, my_pw = 0.f;
+  my_idx = 0;
+  selmask = 0ull;
+  for (int j = 0; j < k; ++j) {
+    // ties keep the lower index: within a lane expert `lane` is below `lane + 32`, across lanes every `lane`
+    // candidate is below every `lane + 32` one, and the lowest lane is the lowest index
+    const unsigned key = key0 >= key1 ? key0 : key1;
+    const unsigned best = __reduce_max_sync(FULL, key);
+    int win;
+    if (!two) {
+      win = __ffs(__ballot_sync(FULL, key0 == best)) - 1;
+    } else {
+      const unsigned b0 = __ballot_sync(FULL, key0 == best), b1 = __ballot_sync(FULL, key1 == best);
+      win = b0 ? __ffs(b0) - 1 : 31 + __ffs(b1);
+    }
+    if (win == lane) key0 = 0u;
+    if (win == lane + 32) key1 = 0u;
+    const float bv = f32_unkey(best);
+    if (j == 0) m = bv;
+    const float pw = expf(bv - m);
+    wtot += pw;
+    selmask |= 1ull << win;
+    if (lane == j) my_pw = pw, my_idx = win;
+  }
+  my_w = my_pw / wtot;
+  if (probs_out || !renorm) {
+    const float p0 = has0 ? expf(l0 - m) : 0.f, p1 = has1 ? expf(l1 - m) : 0.f;
+    const float inv_sum = 1.0f / warp_sum(p0 + p1);
+    if (probs_out) {
+      if (has0) probs_out[lane] = p0 * inv_sum;
+      if (has1) probs_out[lane + 32] = p1 * inv_sum;
+    }
+    if (!renorm) my_w = my_pw * inv_sum;
+  }
+}
+
 __device__ __forceinline__ void warp_route_finish(float l0, float l1, int E, int k, int renorm, int lane,
                                                   int32_t* __restrict__ idx_out, float* __restrict__ w_out,
                                                   float* __restrict__ probs_out) {
-  const unsigned FULL = 0xffffffffu;
-  const float NEG = -3.402823466e38f;
-  const bool has0 = lane < E, has1 = lane + 32 < E;
-  const float m = f32_unkey(__reduce_max_sync(FULL, f32_key(fmaxf(has0 ? l0 : NEG, has1 ? l1 : NEG))));
-  const float p0 = has0 ? expf(l0 - m) : 0.f, p1 = has1 ? expf(l1 - m) : 0.f;
-  const float inv_sum = 1.0f / warp_sum(p0 + p1);
-  if (probs_out) {
-    if (has0) probs_out[lane] = p0 * inv_sum;
-    if (has1) probs_out[lane + 32] = p1 * inv_sum;
-  }
-  bool free0 = has0, free1 = has1;
-  float my_w = 0.f, wtot = 0.f;  // lane j keeps the j-th selected weight
-  int my_idx = 0;
-  for (int j = 0; j < k; ++j) {
-    // this lane's best remaining candidate (its lower index first, so ties keep the lower index)
-    float v = NEG;
-    int id = 0x7fffffff;
-    if (free0) v = l0, id = lane;
-    if (free1 && (!free0 || l1 > v)) v = l1, id = lane + 32;
-    const unsigned key = id != 0x7fffffff ? f32_key(v) : 0u;
-    const unsigned best = __reduce_max_sync(FULL, key);
-    const int win = (int)__reduce_min_sync(FULL, (unsigned)((key == best) ? id : 0x7fffffff));
-    if (win == lane) free0 = false;
-    if (win == lane + 32) free1 = false;
-    const float pw = expf(f32_unkey(best) - m) * inv_sum;
-    wtot += pw;
-    if (lane == j) my_w = pw, my_idx = win;
-  }
+  int my_idx;
+  float my_w;
+  unsigned long long selmask;
+  warp_route_top(l0, l1, E, k, renorm, lane, probs_out, my_idx, my_w, selmask);
   if (lane < k) {
     idx_out[lane] = my_idx;
-    w_out[lane] = renorm ? my_w / wtot : my_w;
+    w_out[lane] = my_w;
   }
 }
 

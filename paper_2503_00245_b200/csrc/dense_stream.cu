@@ -658,14 +658,18 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   const int NS = P.n_stages;
   DeviceState* const st = P.st;
   const int n_pairs = P.T * P.k;
-  const bool fused1 = P.fused_route && P.T == 1;  // one token: the router is spread over the whole CTA
-  constexpr bool kAllX = V >= V_MMA_BF16_S;       // several tokens: every token row is staged once
+  // The variant fixes whether the launch has one token (V_T1, V_COLS) or several (the others): each variant is
+  // compiled without the other case's prologue.
+  constexpr bool kAllX = V >= V_MMA_BF16_S;                 // several tokens: every token row is staged once
+  const bool fused1 = !kAllX && P.fused_route && P.T == 1;  // one token: the router is spread over the whole CTA
+  const bool given1 = !kAllX && P.given1;
 
   // ------------------------------------------------------------------ prologue
   // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as this one's CTAs
   // leave their SMs (its set-up then overlaps this kernel's last CTAs); this kernel in turn reads nothing a
   // predecessor may have written (x, routing, accumulators) before griddepcontrol.wait below.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  uint64_t stream_policy = 0;     // the producer thread's cache hint for the streamed weights
   if (tid == kConsumerThreads) {  // the producer thread sets up the barriers
     for (int i = 0; i < NS; ++i) {
       mbar_init(&sm.full[i], 1);
@@ -680,6 +684,12 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     sm.abort = 0;
     sm.last = 0;
     sm.zero16[0] = sm.zero16[1] = sm.zero16[2] = sm.zero16[3] = 0u;
+    stream_policy = l2_policy_evict_first();
+    if (fused1) {  // one token: k active experts with one slot each, whatever the router will select
+      for (int i = 0; i <= P.k; ++i) sm.act_off[i] = i;
+      for (int i = 0; i < P.k; ++i) sm.slot_tok[i] = 0;
+      sm.n_act = P.k;
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (fused1 && !P.ex.h_in) {
       // one token: every pass reads token row 0, so the first pass's copy of x can start before the routing
@@ -694,7 +704,11 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     }
   }
   PassIt pit;
+  Pass ps;
+  bool pass_known = false;
   if (fused1) pass_split((unsigned)P.k, P.f, pit);  // a single token has k active experts: known before the routing
+  // the host may know the slot of routing entry `lane`'s expert (offload cache); read before anything waits
+  const int given_slot = lane < MOE_MAX_TOPK ? P.ex.slot_of_entry[lane] : -1;
   // the router's weights do not depend on any earlier kernel: the first group of eight experts is fetched
   // before the dependency wait, so its DRAM latency overlaps the predecessor's tail
   // (input features per thread in the router: 4 cover d <= 1024, the shapes of these variants)
@@ -802,40 +816,54 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     // token row 0 was written by the consumer threads (input formed from h): it counts as landed
     if (from_h && tid == kConsumerThreads) mbar_arrive(&sm.xfull[0]);
     if (warp == 0) {
+      // This warp alone stands between the logits and the first weight copy: everything below stays in registers.
+      // The eight warps' partial logits are fetched together and summed in a fixed tree.
       float l0 = bias0, l1 = bias1;
-      if (lane < P.E)
-        for (int w = 0; w < kWarps; ++w) l0 += sm.rlog[w][lane];
-      if (lane + 32 < P.E)
-        for (int w = 0; w < kWarps; ++w) l1 += sm.rlog[w][lane + 32];
-      if (P.ex.use_forced)
+      if (lane < P.E) {
+        float v[kWarps];
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) v[w] = sm.rlog[w][lane];
+        l0 += ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+      }
+      if (lane + 32 < P.E) {
+        float v[kWarps];
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) v[w] = sm.rlog[w][lane + 32];
+        l1 += ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+      }
+      int e = 0;
+      float wv = 0.f;
+      unsigned long long selmask = 0ull;
+      if (P.ex.use_forced) {
         warp_route_forced(l0, l1, P.E, P.k, P.renorm, lane, P.ex.forced, sm.stage_e, sm.stage_w);
-      else
-        warp_route_finish(l0, l1, P.E, P.k, P.renorm, lane, sm.stage_e, sm.stage_w, nullptr);
-      __syncwarp();
-      // the k selected experts in ascending order are the active experts, one slot (token 0) each
+        __syncwarp();
+        if (lane < P.k) e = sm.stage_e[lane], wv = sm.stage_w[lane];
+        const unsigned lo = __reduce_or_sync(0xffffffffu, (lane < P.k && e < 32) ? 1u << e : 0u);
+        const unsigned hi = __reduce_or_sync(0xffffffffu, (lane < P.k && e >= 32) ? 1u << (e - 32) : 0u);
+        selmask = (unsigned long long)lo | ((unsigned long long)hi << 32);
+      } else {
+        warp_route_top(l0, l1, P.E, P.k, P.renorm, lane, nullptr, e, wv, selmask);
+      }
+      // the k selected experts in ascending order are the active experts, one slot (token 0) each; act_off,
+      // slot_tok and n_act do not depend on the selection and were written in the prologue
       if (lane < P.k) {
-        const int e = sm.stage_e[lane];
-        int rank = 0;
-        for (int i = 0; i < P.k; ++i) rank += (sm.stage_e[i] < e);
-        const int given = P.ex.slot_of_entry[lane];  // the host may know the slot (offload cache)
-        const int sl = given >= 0 ? given : (P.expert_slot ? P.expert_slot[e] : e);
+        const int rank = __popcll(selmask & ((1ull << e) - 1ull));
+        const int sl = given_slot >= 0 ? given_slot : (P.expert_slot ? P.expert_slot[e] : e);
         if (sl < 0) flag_error(st, MOE_ERR_STATE, 0x301u);
         sm.act_e[rank] = e;
         sm.act_slot[rank] = sl < 0 ? 0 : sl;
-        sm.act_off[rank] = rank;
-        sm.slot_tok[rank] = 0;
-        sm.slot_w[rank] = sm.stage_w[lane];
+        sm.slot_w[rank] = wv;
         if (blockIdx.x == 0) {
           if (P.topk_idx) P.topk_idx[lane] = e;
-          if (P.topk_w) P.topk_w[lane] = sm.stage_w[lane];
+          if (P.topk_w) P.topk_w[lane] = wv;
         }
       }
-      if (lane == 0) {
-        sm.act_off[P.k] = P.k;
-        sm.n_act = P.k;
-      }
+    } else {
+      // meanwhile the other warps work out this CTA's share: it depends on the number of active experts only
+      pass_init(sm, P.f, pit, true, (unsigned)P.k);
+      pass_known = true;
     }
-  } else if (P.fused_route) {
+  } else if (kAllX && P.fused_route) {
     // several tokens, E a multiple of 8 (Eq. 2, Eq. 3); every CTA routes all tokens.  A thread owns the input
     // features tid, tid + 256, ...: their router rows are fetched once and serve every token; the tokens go
     // four at a time so that all their loads are in flight together.
@@ -905,7 +933,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
       }
     }
-  } else if (P.given1) {
+  } else if (given1) {
     // one token, routing given: the entries of topk_idx / topk_w this launch was asked for, ascending by expert
     if (warp == 0) {
       const bool mine = lane < P.k && ((P.ex.sel_mask >> lane) & 1u);
@@ -936,14 +964,14 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         if (bad) flag_error(st, MOE_ERR_STATE, 0x302u);
       }
     }
-  } else if (P.mode == 0 && warp == 0) {
+  } else if (kAllX && P.mode == 0 && warp == 0) {
     for (int p = lane; p < n_pairs; p += 32) {
       sm.stage_e[p] = P.topk_idx[p];
       sm.stage_w[p] = P.topk_w[p];
     }
   }
-  __syncthreads();
-  if (warp == 0 && !fused1 && !P.given1 && P.mode == 0) {
+  if (!fused1) __syncthreads();  // (one token with the router fused: nothing happens between this barrier and the next)
+  if (kAllX && warp == 0 && !fused1 && !given1 && P.mode == 0) {
     // routing products -> active experts and their slots (same numbering as moe_permute): lane e works for
     // experts e and e + 32
     const int n = n_pairs, E = P.E;
@@ -1054,8 +1082,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   }
   __syncthreads();
 
-  pass_init(sm, P.f, pit, fused1, (unsigned)P.k);
-  Pass ps;
+  if (!pass_known) pass_init(sm, P.f, pit, fused1, (unsigned)P.k);
   RingPos rp{0, 0u, 0};
 
   if (warp == kProducerWarp) {
@@ -1064,15 +1091,14 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     const uint32_t row_bytes = (uint32_t)(3 * P.d * 2);
     const uint32_t xrow_bytes = (uint32_t)P.d * (P.x_is_bf16 ? 2u : 4u);
     bool ok = true;
-    const uint64_t stream_policy = l2_policy_evict_first();
     int pn = 0, pn_issued = 0;
-    int last_idx[2] = {-1, -1};  // ring index of the last stage of the pass that used xs[b] before
+    int last_idx0 = -1, last_idx1 = -1;  // ring index of the last stage of the pass that used xs[0 / 1] before
     int known_free = -1;         // every ring index <= known_free has been released by the consumers
     unsigned copy_mask = 0;
     while (ok && next_pass(sm, P.f, pit, ps)) {
       const int b = pn & 1;
-      if (!kAllX && last_idx[b] > known_free) {
-        const int L = last_idx[b];
+      if (!kAllX && (b ? last_idx1 : last_idx0) > known_free) {
+        const int L = b ? last_idx1 : last_idx0;
         if (!mbar_wait(&sm.freeb[L % NS], (unsigned)(L / NS) & 1u)) {
           set_abort(st, sm, 0x331u);
           ok = false;
@@ -1143,7 +1169,10 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         src += bytes;
         rp.advance(NS);
       }
-      last_idx[b] = rp.n - 1;
+      if (b)
+        last_idx1 = rp.n - 1;
+      else
+        last_idx0 = rp.n - 1;
       ++pn;
     }
     if ((fused1 || kAllX) && pn_issued == 0) (void)mbar_wait(&sm.xfull[0], 0u);  // the early copy of x must land
@@ -1207,8 +1236,12 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     int slice = (int)old - (int)(G - K);
     if (slice >= 0 && old != G - 1u) {
       const long long t0 = clock64();
-      while (ld_acquire64(&st->done_total) < target) {
-        if (clock64() - t0 > P.fin_wait_budget || sm.abort || ld_acquire(&st->status) != 0u) {
+      for (;;) {
+        // both words in one round trip: the status load is not ordered against the counter's, it only ends a wait
+        // that an error elsewhere has made pointless
+        const unsigned err = ld_relaxed(&st->status);
+        if (ld_acquire64(&st->done_total) >= target) break;
+        if (clock64() - t0 > P.fin_wait_budget || sm.abort || err != 0u) {
           flag_error(st, MOE_ERR_TIMEOUT, 0x340u);  // (keeps an earlier error code if one is set)
           slice = -1;
           break;
@@ -1225,7 +1258,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     const long long total = (long long)rows * P.d;
     const long long per = (total + K - 1) / K;
     const long long lo = per * slice, hi = lo + per < total ? lo + per : total;
-    const bool good = ld_acquire(&st->status) == 0u;
+    // (ordered after the full arrival count by the barrier above; an acquire here would hold the loads below back)
+    const unsigned err_seen = ld_relaxed(&st->status);
     // four outputs per thread at a time: all their copies are fetched in one round trip, then summed,
     // converted, stored, and the copies zeroed
     for (long long i0 = lo + tid; i0 < hi; i0 += 4 * kConsumerThreads) {
@@ -1247,7 +1281,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           v += part[j][c];
           if (c < P.acc_copies) P.acc[(size_t)c * P.acc_copy_stride + i] = 0;
         }
-        if (!good) continue;
+        if (err_seen != 0u) continue;
         const float fv = (float)((double)v * kFixInv);
         if (P.mode == 1)
           P.out_slots[i] = fv;
