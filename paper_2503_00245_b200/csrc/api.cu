@@ -198,7 +198,12 @@ int moe_seed_arrival_counter(moe_ctx* ctx, unsigned long long value, void* strea
   if (!ctx) return MOE_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   ctx->h_state->done_total = value;
+  // one-token launches count arrivals in the accumulator words instead: a counter that is out of step with the
+  // grid size makes them wait for one arrival more than a launch has
+  ctx->h_state->tail_bias = (value % (unsigned long long)ctx->sm_count) != 0ull ? 1u : 0u;
   MOE_CUDA_TRY(cudaMemcpyAsync(&ctx->d_state->done_total, &ctx->h_state->done_total, sizeof(unsigned long long),
+                               cudaMemcpyHostToDevice, s));
+  MOE_CUDA_TRY(cudaMemcpyAsync(&ctx->d_state->tail_bias, &ctx->h_state->tail_bias, sizeof(unsigned int),
                                cudaMemcpyHostToDevice, s));
   MOE_CUDA_TRY(cudaStreamSynchronize(s));
   return MOE_OK;

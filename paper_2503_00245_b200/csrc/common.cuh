@@ -39,7 +39,10 @@ struct DeviceState {
   // dense streaming kernel, one token: next stage (4 hidden units) of each active expert that no CTA has taken yet;
   // the finalisers leave zeros
   unsigned int stage_ctr[MOE_MAX_TOPK];
-  unsigned int pad3[20];
+  // dense streaming kernel, one token: added to the arrivals an accumulator word waits for (0; the diagnostics
+  // hook sets 1, so that the wait runs out)
+  unsigned int tail_bias;
+  unsigned int pad3[19];
 };
 
 }  // namespace cosmoe
@@ -255,6 +258,11 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
 __device__ __forceinline__ unsigned ld_relaxed(const unsigned* p) {
   unsigned v;
   asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned long long ld_relaxed64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {

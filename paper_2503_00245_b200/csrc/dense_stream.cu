@@ -42,6 +42,13 @@ constexpr int kMaxSlots = MOE_STREAM_MAX_TOKENS * MOE_MAX_TOPK;
 constexpr int kFinalizers = 8;  // CTAs that share the conversion of the sums into the output
 constexpr float kFixScale = 68719476736.0f;      // 2^36
 constexpr double kFixInv = 1.0 / 68719476736.0;
+// One token, one launch per layer: the accumulator words also count the CTAs that have added to them.  A CTA adds
+// (sum * 2^32 rounded) * 2^8 + 1, so the low 8 bits of a word are the number of arrivals (at most 255 per word)
+// and the rest is the sum in units of 2^-32 (|sum| < 2^23): whoever reads a word with the full count has the
+// final sum in hand -- no arrival counter, no fence between the sums and the count, no second read.
+constexpr float kFixScaleCnt = 4294967296.0f;  // 2^32
+constexpr double kFixInvCnt = 1.0 / 4294967296.0;
+constexpr int kCntBits = 8;
 
 struct DenseParams {
   int T, k, E, d, f, mode, x_is_bf16, renorm, fused_route;
@@ -68,6 +75,7 @@ struct DenseParams {
   int f_full;                  // hidden units per expert in memory (f may be a sub-range of them, starting at ex.unit_lo)
   int given1;                  // one token, routing taken from topk_idx / topk_w (possibly a subset of its entries)
   int dyn;                     // one token, d > 1024: stages are handed out from per-expert counters (see consume_pass_cols)
+  int counted;                 // one token, whole layer in this launch: arrivals are counted in the accumulator words
   DenseExtra ex;
 };
 
@@ -317,7 +325,8 @@ __device__ __forceinline__ bool consume_pass_t1(const DenseParams& P, Smem& sm, 
       float v = 0.f;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) v += wpart[(size_t)w * d + i];
-      atomicAdd(dst + i, (unsigned long long)__float2ll_rn(v * kFixScale));
+      atomicAdd(dst + i, P.counted ? ((unsigned long long)__float2ll_rn(v * kFixScaleCnt) << kCntBits) + 1ull
+                                   : (unsigned long long)__float2ll_rn(v * kFixScale));
     }
   }
   return consumer_sync(sm, cpar, lane);  // wpart may be rewritten by the next pass
@@ -561,6 +570,7 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
   const int mychunk = cw0 + lane;
   const bool owner = mychunk < cw1;
   const int cclamp = owner ? mychunk : cw0;
+  const float fix = P.counted ? kFixScaleCnt : kFixScale;
   float acc[8];
   long long iacc[8];  // dynamic hand-out: fixed-point sums, so that the result does not depend on which CTA took which stage
 #pragma unroll
@@ -627,7 +637,7 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
     }
     if (P.dyn) {  // a stage's sum depends on the stage alone; integer addition across stages is associative
 #pragma unroll
-      for (int j = 0; j < 8; ++j) iacc[j] += __float2ll_rn(acc[j] * kFixScale), acc[j] = 0.f;
+      for (int j = 0; j < 8; ++j) iacc[j] += __float2ll_rn(acc[j] * fix), acc[j] = 0.f;
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.freeb[rp.slot]);
@@ -638,7 +648,10 @@ __device__ __forceinline__ bool consume_pass_cols(const DenseParams& P, Smem& sm
     unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) +
                               (size_t)(blockIdx.x % P.acc_copies) * P.acc_copy_stride + (size_t)rowi * d + mychunk * 8;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) atomicAdd(dst + j, (unsigned long long)(P.dyn ? iacc[j] : __float2ll_rn(acc[j] * kFixScale)));
+    for (int j = 0; j < 8; ++j) {
+      const long long v = P.dyn ? iacc[j] : __float2ll_rn(acc[j] * fix);
+      atomicAdd(dst + j, P.counted ? ((unsigned long long)v << kCntBits) + 1ull : (unsigned long long)v);
+    }
   }
   return true;
 }
@@ -706,6 +719,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   PassIt pit;
   Pass ps;
   bool pass_known = false;
+  int pre_stage = 0;  // producer thread: 1 = the first stage's barrier already expects its bytes (see below)
   if (fused1) pass_split((unsigned)P.k, P.f, pit);  // a single token has k active experts: known before the routing
   // the host may know the slot of routing entry `lane`'s expert (offload cache); read before anything waits
   const int given_slot = lane < MOE_MAX_TOPK ? P.ex.slot_of_entry[lane] : -1;
@@ -862,6 +876,18 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       // meanwhile the other warps work out this CTA's share: it depends on the number of active experts only
       pass_init(sm, P.f, pit, true, (unsigned)P.k);
       pass_known = true;
+      // The producer thread readies its first stage now: which hidden units it covers depends on the launch shape
+      // only, so the stage's barrier can be armed here and the copy issued the moment the expert is known.
+      // (a CTA that works for one expert; with dynamic hand-out the first stage comes from its static share)
+      if (!kAllX && tid == kConsumerThreads && pit.cta_c > 0 &&
+          (!P.dyn || (P.f + kRows - 1) / kRows >= 2 * pit.cta_c) && next_pass(sm, P.f, pit, ps)) {
+        const int n_st = (P.f + kRows - 1) / kRows;
+        const int cur = P.dyn ? pit.cta_j * (n_st / (2 * pit.cta_c)) : 0;
+        const int nrows = P.dyn ? min(kRows, P.f - cur * kRows) : min(kRows, ps.rb - ps.ra);
+        if (P.dyn) sm.stage_n[0] = nrows;
+        mbar_arrive_expect_tx(&sm.full[0], (uint32_t)nrows * (uint32_t)(3 * P.d * 2));
+        pre_stage = 1;
+      }
     }
   } else if (kAllX && P.fused_route) {
     // several tokens, E a multiple of 8 (Eq. 2, Eq. 3); every CTA routes all tokens.  A thread owns the input
@@ -1095,7 +1121,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     int last_idx0 = -1, last_idx1 = -1;  // ring index of the last stage of the pass that used xs[0 / 1] before
     int known_free = -1;         // every ring index <= known_free has been released by the consumers
     unsigned copy_mask = 0;
-    while (ok && next_pass(sm, P.f, pit, ps)) {
+    while (ok && (pre_stage == 1 || next_pass(sm, P.f, pit, ps))) {
       const int b = pn & 1;
       if (!kAllX && (b ? last_idx1 : last_idx0) > known_free) {
         const int L = b ? last_idx1 : last_idx0;
@@ -1123,7 +1149,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       // expert's stages (4 hidden units each) statically and then draws single stages from the expert's counter until
       // none is left.  A stage with zero units tells the consumers that the pass is over.
       const int n_st = (P.f + kRows - 1) / kRows;
-      const int dyn_s0 = P.dyn ? (int)((long long)n_st / (2 * pit.cta_c)) : 0;
+      const int dyn_s0 = P.dyn ? n_st / (2 * pit.cta_c) : 0;
       int dyn_next = pit.cta_j * dyn_s0;
       const int dyn_stat_end = dyn_next + dyn_s0, dyn_base = pit.cta_c * dyn_s0;
       for (int row = ps.ra; P.dyn || row < ps.rb; row += kRows) {
@@ -1134,6 +1160,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
         const int nrows = P.dyn ? (cur < 0 ? 0 : min(kRows, P.f - cur * kRows)) : min(kRows, ps.rb - row);
         const uint32_t bytes = (uint32_t)nrows * row_bytes;
+        const bool armed = pre_stage == 1;  // first stage of the launch: ring slot 0, its barrier already expects `bytes`
+        pre_stage = 2;
         if (rp.n >= NS) {
           if (!mbar_wait(&sm.freeb[rp.slot], rp.par ^ 1u)) {
             set_abort(st, sm, 0x330u);
@@ -1147,7 +1175,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           break;
         }
         if (P.dyn) {
-          sm.stage_n[rp.slot] = nrows;
+          if (!armed) sm.stage_n[rp.slot] = nrows;
           if (nrows == 0) {  // no stage left: the consumers leave on this one
             mbar_arrive(&sm.full[rp.slot]);
             rp.advance(NS);
@@ -1156,8 +1184,10 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           src = reinterpret_cast<const unsigned char*>(P.gud) +
                 ((size_t)sm.act_slot[ps.ai] * P.f_full + P.ex.unit_lo + (size_t)cur * kRows) * row_bytes;
         }
-        fence_proxy_async_smem();
-        mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
+        if (!armed) {
+          fence_proxy_async_smem();
+          mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
+        }
         if (P.use_mma) {  // one copy per hidden unit: the units are padded apart in shared memory
           for (uint32_t o = 0, u = 0; o < bytes; o += row_bytes, ++u)
             bulk_g2s_hint(ring + (size_t)rp.slot * P.stage_bytes + (size_t)u * P.unit_stride, src + o, row_bytes,
@@ -1192,6 +1222,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
 
   // ===================================================================== consumers
   unsigned cpar = 0;
+  int passes_done = 0;
   {
     bool ok = true;
     int pn = 0;
@@ -1217,10 +1248,69 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         ok = consume_pass_mma<false, 8, 16>(P, sm, ps, ring, xsb, rp, warp, lane);
       ++pn;
     }
+    passes_done = ok ? pn : -1;
   }
   // ------------------------------------------------------------------ all partial sums are out
   // (after an expired wait the warps may be out of step with this barrier: then it can expire too; the
   // status word is already set and nobody finalises)
+  if (!kAllX && P.counted) {
+    // ---------------------------------------------------------------- one token: the words count their arrivals
+    // Every CTA adds to every output element exactly once (a CTA without a share adds zeros), into the copy
+    // blockIdx % copies; CTA b finishes the elements [b d / G, (b + 1) d / G): thread (element, copy) polls its
+    // word until the count is full, the copies of an element are summed over neighbouring lanes, the sum is
+    // converted and stored and the words are left zero.  The wait is bounded like every other.
+    const int G = (int)gridDim.x, b = (int)blockIdx.x, d = P.d, copies = P.acc_copies;  // copies: a power of two <= 32
+    if (passes_done < 0) return;  // an expired wait: the status word is set, the pollers elsewhere give up on it
+    if (passes_done == 0) {
+      unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.acc) + (size_t)(b % copies) * P.acc_copy_stride;
+      for (int i = tid; i < d; i += kConsumerThreads) atomicAdd(dst + i, 1ull);
+    }
+    const int lo = (int)((long long)b * d / G), hi = (int)((long long)(b + 1) * d / G);
+    const int per_round = kConsumerThreads / copies;  // elements handled at a time
+    const unsigned bias = ld_relaxed(&st->tail_bias);  // 0 (the diagnostics hook: 1, a count the launch never reaches)
+    for (int e0 = lo; e0 < hi; e0 += per_round) {
+      const int el = e0 + tid / copies, c = tid % copies;
+      const bool mine = el < hi;
+      if (__ballot_sync(0xffffffffu, mine) == 0u) continue;  // (whole warps leave together: the shuffles below are warp-wide)
+      const unsigned expect = (unsigned)((G - c + copies - 1) / copies) + bias;
+      unsigned long long* word = reinterpret_cast<unsigned long long*>(P.acc) + (size_t)c * P.acc_copy_stride + (mine ? el : lo);
+      unsigned long long v = 0ull;
+      bool ok = true;
+      const long long t0 = clock64();
+      for (unsigned spins = 0;; ++spins) {
+        v = ld_relaxed64(word);
+        const bool full = !mine || (unsigned)(v & ((1ull << kCntBits) - 1ull)) == expect;
+        if (__all_sync(0xffffffffu, full)) break;
+        const bool give_up = (spins & 7u) == 7u && (clock64() - t0 > P.fin_wait_budget || ld_relaxed(&st->status) != 0u);
+        if (__any_sync(0xffffffffu, give_up)) {
+          ok = false;
+          break;
+        }
+      }
+      if (!ok) {
+        if (lane == 0) flag_error(st, MOE_ERR_TIMEOUT, 0x341u);  // (keeps an earlier error code if one is set)
+        break;
+      }
+      long long sum = (long long)v >> kCntBits;  // arithmetic shift: the count falls off, the sum keeps its sign
+      if (!mine) sum = 0;
+      for (int o = 1; o < copies; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (mine) {
+        *word = 0ull;
+        if (c == 0) {
+          const float fv = (float)((double)sum * kFixInvCnt);
+          if (P.ex.resid)
+            P.ex.resid[el] += fv;  // h += y
+          else if (P.x_is_bf16)
+            ((__nv_bfloat16*)P.y)[el] = __float2bfloat16_rn(fv);
+          else
+            ((float*)P.y)[el] = fv;
+        }
+      }
+      // CTA 0's first element is complete: every CTA has streamed its last stage, nobody draws stages any more
+      if (b == 0 && e0 == lo && tid < MOE_MAX_TOPK) st->stage_ctr[tid] = 0u;
+    }
+    return;
+  }
   bool fin = consumer_sync(sm, cpar, lane);
   if (!P.ex.finalize) return;  // a later launch of the group adds its share and finalises
   // The last kFinalizers CTAs to arrive turn the fixed-point sums into the output, one slice each, and leave
@@ -1378,6 +1468,13 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
            G >= c.top_k && c.d_ff >= 8 * G)
               ? 1
               : 0;
+  // one token and the whole layer in this launch: arrivals are counted in the accumulator words themselves
+  P.counted = (mode == 0 && T == 1 && P.ex.finalize && P.ex.unit_cnt == 0 &&
+               (P.ex.sel_mask & ((1u << c.top_k) - 1u)) == (1u << c.top_k) - 1u && G >= c.top_k && c.top_k <= 16 &&
+               P.acc_copies >= 1 && P.acc_copies <= 32 && (P.acc_copies & (P.acc_copies - 1)) == 0 &&
+               (G + P.acc_copies - 1) / P.acc_copies + 1 < (1 << kCntBits))
+                  ? 1
+                  : 0;
   int rc;
   switch (v) {
     case V_T1: rc = launch_variant<V_T1>(P, G, smem, s); break;
