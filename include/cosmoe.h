@@ -121,8 +121,10 @@ int moe_workspace_bytes(const moe_config* cfg, int32_t T, size_t* bytes);
  * moe_seed_arrival_counter: overwrites the ctx's arrival counter (which normally runs over launches and is a
  * multiple of the grid size between calls) and waits for `stream`.  Seeded with grid size - 1, the next launch's
  * arrivals straddle a multiple of the grid size, so most of its finalisers wait for a count that launch never
- * reaches: with a short budget they give up, every CTA having streamed its share and exited normally.  The
- * output of such a call is undefined; moe_check reports MOE_ERR_TIMEOUT and re-arms the state.               */
+ * reaches: with a short budget they give up, every CTA having streamed its share and exited normally.  (A
+ * one-token launch counts arrivals in its accumulator words instead; a value that is not a multiple of the grid
+ * size makes those words wait for one arrival more than the launch has, to the same effect.)  The output of
+ * such a call is undefined; moe_check reports MOE_ERR_TIMEOUT and re-arms the state.                          */
 int moe_set_finaliser_wait(moe_ctx* ctx, long long cycles);
 int moe_seed_arrival_counter(moe_ctx* ctx, unsigned long long value, void* stream);
 /* Kernels launched by hot calls on this ctx since creation (for accounting). */

@@ -3,8 +3,10 @@
 The dense streaming kernel's last CTAs wait (bounded) for the arrival counter before they turn the partial sums
 into the output: each waits until the count reaches the next multiple of the grid size.  The counter is seeded
 with grid size - 1, so the launch's arrivals straddle a multiple: all but one finaliser wait for a count this
-launch never reaches, and with the budget cut to half a millisecond they give up.  Every CTA has streamed its
-share, added its sums and exits normally; the finalisers that gave up flag MOE_ERR_TIMEOUT.
+launch never reaches, and with the budget cut to half a millisecond they give up.  (A one-token launch counts
+its arrivals in the accumulator words themselves; the same call makes those words wait for one arrival more than
+the launch has.)  Every CTA has streamed its share, added its sums and exits normally; the finalisers that gave
+up flag MOE_ERR_TIMEOUT.
 Checked: moe_check reports the time-out, clears it and re-arms the ctx's state (arrival counter, accumulators),
 and the next ordinary call is bit-identical to a fresh ctx's and matches the CPU checker."""
 import numpy as np
