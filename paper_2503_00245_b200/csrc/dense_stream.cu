@@ -39,6 +39,7 @@ constexpr int kMaxN = 8;       // tokens of one expert handled per pass over its
 constexpr int kMaxStages = 8;
 constexpr int kXIters = 8;     // 16-byte chunks of x per lane: d <= 2048
 constexpr int kMaxSlots = MOE_STREAM_MAX_TOKENS * MOE_MAX_TOPK;
+constexpr int kPreStages = 3;   // one token: stages whose copies go out before the general issue loop starts
 constexpr int kFinalizers = 8;  // CTAs that share the conversion of the sums into the output
 constexpr float kFixScale = 68719476736.0f;      // 2^36
 constexpr double kFixInv = 1.0 / 68719476736.0;
@@ -719,7 +720,10 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   PassIt pit;
   Pass ps;
   bool pass_known = false;
-  int pre_stage = 0;  // producer thread: 1 = the first stage's barrier already expects its bytes (see below)
+  // producer thread, one token: its first pass is fetched (pre_stage 1) and the barriers of that pass's first pre_n
+  // stages already expect their bytes before the routing is known; pre_off: where those stages start inside an expert
+  int pre_stage = 0, pre_n = 0;
+  size_t pre_off = 0;
   if (fused1) pass_split((unsigned)P.k, P.f, pit);  // a single token has k active experts: known before the routing
   // the host may know the slot of routing entry `lane`'s expert (offload cache); read before anything waits
   const int given_slot = lane < MOE_MAX_TOPK ? P.ex.slot_of_entry[lane] : -1;
@@ -876,16 +880,22 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       // meanwhile the other warps work out this CTA's share: it depends on the number of active experts only
       pass_init(sm, P.f, pit, true, (unsigned)P.k);
       pass_known = true;
-      // The producer thread readies its first stage now: which hidden units it covers depends on the launch shape
-      // only, so the stage's barrier can be armed here and the copy issued the moment the expert is known.
-      // (a CTA that works for one expert; with dynamic hand-out the first stage comes from its static share)
-      if (!kAllX && tid == kConsumerThreads && pit.cta_c > 0 &&
-          (!P.dyn || (P.f + kRows - 1) / kRows >= 2 * pit.cta_c) && next_pass(sm, P.f, pit, ps)) {
+      // The producer thread readies its first stages now: which hidden units they cover depends on the launch shape
+      // only, so their barriers are armed here and, once the expert is known, the copies go out from a loop of a
+      // few instructions -- the general issue loop below is cold code at that point (its instructions come from L2,
+      // a few hundred cycles per line), and warms up while these copies are on their way.
+      // (a CTA that works for one expert; with dynamic hand-out the first stages come from its static share)
+      if (!kAllX && tid == kConsumerThreads && pit.cta_c > 0 && next_pass(sm, P.f, pit, ps)) {
         const int n_st = (P.f + kRows - 1) / kRows;
-        const int cur = P.dyn ? pit.cta_j * (n_st / (2 * pit.cta_c)) : 0;
-        const int nrows = P.dyn ? min(kRows, P.f - cur * kRows) : min(kRows, ps.rb - ps.ra);
-        if (P.dyn) sm.stage_n[0] = nrows;
-        mbar_arrive_expect_tx(&sm.full[0], (uint32_t)nrows * (uint32_t)(3 * P.d * 2));
+        const int dyn_s0 = P.dyn ? n_st / (2 * pit.cta_c) : 0;
+        const int first = P.dyn ? pit.cta_j * dyn_s0 * kRows : ps.ra;  // first hidden unit this CTA streams
+        const int whole = P.dyn ? min(dyn_s0, (P.f - first) / kRows) : (ps.rb - ps.ra) / kRows;  // stages of kRows units
+        pre_n = min(min(kPreStages, NS), whole);
+        for (int i = 0; i < pre_n; ++i) {
+          if (P.dyn) sm.stage_n[i] = kRows;
+          mbar_arrive_expect_tx(&sm.full[i], (uint32_t)kRows * (uint32_t)(3 * P.d * 2));
+        }
+        pre_off = (size_t)(P.ex.unit_lo + first) * (size_t)(3 * P.d * 2);
         pre_stage = 1;
       }
     }
@@ -1121,7 +1131,15 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     int last_idx0 = -1, last_idx1 = -1;  // ring index of the last stage of the pass that used xs[0 / 1] before
     int known_free = -1;         // every ring index <= known_free has been released by the consumers
     unsigned copy_mask = 0;
+    if (pre_n > 0) {  // the stages armed before the routing was known: only the expert was missing
+      const unsigned char* src0 = reinterpret_cast<const unsigned char*>(P.gud) +
+                                  (size_t)sm.act_slot[ps.ai] * P.f_full * row_bytes + pre_off;
+      for (int i = 0; i < pre_n; ++i, src0 += kRows * row_bytes)
+        bulk_g2s_hint(ring + (size_t)i * P.stage_bytes, src0, kRows * row_bytes, &sm.full[i], stream_policy);
+    }
     while (ok && (pre_stage == 1 || next_pass(sm, P.f, pit, ps))) {
+      const int skip = pre_stage == 1 ? pre_n : 0;  // stages of this pass that are already on their way
+      pre_stage = 2;
       const int b = pn & 1;
       if (!kAllX && (b ? last_idx1 : last_idx0) > known_free) {
         const int L = b ? last_idx1 : last_idx0;
@@ -1143,16 +1161,20 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
                    (const unsigned char*)P.x + (size_t)sm.slot_tok[slot0 + s] * xrow_bytes, xrow_bytes, &sm.xfull[b]);
       }
       const unsigned char* src = reinterpret_cast<const unsigned char*>(P.gud) +
-                                 ((size_t)sm.act_slot[ps.ai] * P.f_full + P.ex.unit_lo + ps.ra) * row_bytes;
+                                 ((size_t)sm.act_slot[ps.ai] * P.f_full + P.ex.unit_lo + ps.ra + skip * kRows) * row_bytes;
       // Dynamic hand-out (one token, one pass per CTA): the CTAs of an expert do not stream at the same rate -- equal
       // shares end up to 4 us apart at the phone shape -- so a CTA takes half of its equal share of the
       // expert's stages (4 hidden units each) statically and then draws single stages from the expert's counter until
       // none is left.  A stage with zero units tells the consumers that the pass is over.
       const int n_st = (P.f + kRows - 1) / kRows;
       const int dyn_s0 = P.dyn ? n_st / (2 * pit.cta_c) : 0;
-      int dyn_next = pit.cta_j * dyn_s0;
-      const int dyn_stat_end = dyn_next + dyn_s0, dyn_base = pit.cta_c * dyn_s0;
-      for (int row = ps.ra; P.dyn || row < ps.rb; row += kRows) {
+      int dyn_next = pit.cta_j * dyn_s0 + skip;
+      const int dyn_stat_end = pit.cta_j * dyn_s0 + dyn_s0, dyn_base = pit.cta_c * dyn_s0;
+      for (int i = 0; i < skip; ++i) {
+        copy_mask |= 1u << rp.slot;
+        rp.advance(NS);
+      }
+      for (int row = ps.ra + skip * kRows; P.dyn || row < ps.rb; row += kRows) {
         int cur = 0;
         if (P.dyn) {
           cur = dyn_next < dyn_stat_end ? dyn_next++ : dyn_base + (int)atomicAdd(&st->stage_ctr[ps.ai], 1u);
@@ -1160,8 +1182,6 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         }
         const int nrows = P.dyn ? (cur < 0 ? 0 : min(kRows, P.f - cur * kRows)) : min(kRows, ps.rb - row);
         const uint32_t bytes = (uint32_t)nrows * row_bytes;
-        const bool armed = pre_stage == 1;  // first stage of the launch: ring slot 0, its barrier already expects `bytes`
-        pre_stage = 2;
         if (rp.n >= NS) {
           if (!mbar_wait(&sm.freeb[rp.slot], rp.par ^ 1u)) {
             set_abort(st, sm, 0x330u);
@@ -1175,7 +1195,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           break;
         }
         if (P.dyn) {
-          if (!armed) sm.stage_n[rp.slot] = nrows;
+          sm.stage_n[rp.slot] = nrows;
           if (nrows == 0) {  // no stage left: the consumers leave on this one
             mbar_arrive(&sm.full[rp.slot]);
             rp.advance(NS);
@@ -1184,10 +1204,8 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
           src = reinterpret_cast<const unsigned char*>(P.gud) +
                 ((size_t)sm.act_slot[ps.ai] * P.f_full + P.ex.unit_lo + (size_t)cur * kRows) * row_bytes;
         }
-        if (!armed) {
-          fence_proxy_async_smem();
-          mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
-        }
+        fence_proxy_async_smem();
+        mbar_arrive_expect_tx(&sm.full[rp.slot], bytes);
         if (P.use_mma) {  // one copy per hidden unit: the units are padded apart in shared memory
           for (uint32_t o = 0, u = 0; o < bytes; o += row_bytes, ++u)
             bulk_g2s_hint(ring + (size_t)rp.slot * P.stage_bytes + (size_t)u * P.unit_stride, src + o, row_bytes,
