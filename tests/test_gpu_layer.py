@@ -58,6 +58,13 @@ def shape(d, f, E=8, k=2, r=0, xd="bf16", bias="none", cfg_id=8):
     (shape(400, 1280, r=200), 1, 0),                # wearable-WD widths
     (shape(400, 1280, r=200), 64, 0),
     (shape(4096, 512), 4, 0),                       # dense, d_model beyond the streaming kernel: tensor path at small T
+    # one token, accumulator words that count their arrivals: CTAs without a share (fewer hidden units than CTAs per
+    # expert) still have to be counted; one and eight choices change the arrivals a word waits for; fp32 rows
+    (shape(256, 64), 1, 0),
+    (shape(256, 40, E=8, k=1), 1, 0),
+    (shape(1024, 2816, E=8, k=8), 1, 0),
+    (shape(2048, 1024, E=8, k=1, xd="f32"), 1, 0),
+    (shape(256, 512, E=64, k=4), 1, 0),             # two logits per lane in the routing warp
 ])
 def test_layer_forward_matches_checker(sh, T, path):
     lay, t, host = U.build(sh, T, path=path)
