@@ -26,8 +26,10 @@
  *    top_k <= 8.  Anything else: MOE_ERR_UNSUPPORTED, nothing is read or written.
  *    The streaming path of dense experts also needs d_model <= 2048.
  *  - The streaming path sums the CTAs' partial outputs with 64-bit fixed-point atomics
- *    (2^-36 resolution): integer addition is associative, so results do not depend on
- *    the order of arrival and repeated calls are bit-identical.
+ *    (2^-36 resolution, |partial sums| < 2^27; a one-token call of a whole layer keeps the
+ *    number of arrivals in the low bits of the same words: 2^-32 resolution, |sums| < 2^23):
+ *    integer addition is associative, so results do not depend on the order of arrival and
+ *    repeated calls are bit-identical.  Outputs beyond those magnitudes are not supported.
  *
  * Weight layouts.  The mathematical layouts (row-vector convention y = x W) are
  *    w_gate, w_up [E][d][f],  w_down [E][f][d]                       (dense)
