@@ -35,6 +35,7 @@ constexpr int kProducerWarp = kWarps;
 constexpr int kThreads = (kWarps + 1) * 32;
 constexpr int kConsumerThreads = kWarps * 32;
 constexpr int kRows = 4;       // hidden units per stage: kWarps dot products
+constexpr int kRowsWide = 8;   // several tokens at d <= 1024: 8 units per stage fill both the 16 rows and the 8 k-values of the MMAs
 constexpr int kMaxN = 8;       // tokens of one expert handled per pass over its units
 constexpr int kMaxStages = 8;
 constexpr int kXIters = 8;     // 16-byte chunks of x per lane: d <= 2048
@@ -67,6 +68,7 @@ struct DenseParams {
   DeviceState* st;
   long long* acc;
   int stage_bytes, n_stages, xs_bytes;
+  int stage_rows;              // hidden units per stage: kRows, or kRowsWide for several tokens at d <= 1024
   int unit_stride;             // bytes between the hidden units of a stage (3 rows, padded for the MMA passes)
   int use_mma;                 // more than one token: every pass goes through consume_pass_mma
   int wpart_ok;                // shared memory holds the [8][d] merge buffer of the unit-owner passes (d <= 1024)
@@ -87,18 +89,26 @@ struct Smem {
   uint64_t xfull[2];           // token rows of a pass landed in xs[0/1]
   uint64_t cbar;               // barrier over the consumer warps
   int stage_n[kMaxStages];             // dynamic hand-out: hidden units in the stage (0 = no more stages)
-  float gu[kMaxStages][kRows * 2];     // single-token passes at d > 1024: the stage's 8 dot products
-  __align__(16) float red[4][2][kRows * 8][kWarps];  // multi-token passes: [stage index & 3][gate | up][unit * 8 + token][warp]
+  // `red` belongs to the passes with several tokens.  Before the passes, and in launches with one token, the same
+  // bytes hold what only the prologue (or only a single-token pass) needs: with them in the header a launch with 8
+  // tokens at d = 1024 would have room for 3 ring stages instead of 4.
+  union {
+    __align__(16) float red[4][2][kRowsWide * 8][kWarps];  // [stage index & 3][gate | up][unit * 8 + token][warp]
+    struct {
+      float scratch[kWarps * 16 * 16];     // several tokens: the router's partial logits [warp][token][expert]; h = x / rms: 8 sums
+      float rlog[kWarps][MOE_MAX_EXPERTS]; // one token: the router's partial logits
+      float gu[kMaxStages][kRows * 2];     // single-token passes at d > 1024: the stage's 8 dot products
+      int cursor[MOE_MAX_EXPERTS];         // grouping of several tokens
+      int stage_e[kMaxSlots];              // routing as selected, before the grouping
+      float stage_w[kMaxSlots];
+    };
+  };
   __align__(16) uint32_t zero16[4];    // what ldmatrix reads for padding rows
-  float rlog[kWarps][MOE_MAX_EXPERTS];
   int act_e[MOE_MAX_EXPERTS];
   int act_slot[MOE_MAX_EXPERTS];
   int act_off[MOE_MAX_EXPERTS + 1];
   int slot_tok[kMaxSlots];
   float slot_w[kMaxSlots];
-  int cursor[MOE_MAX_EXPERTS];
-  int stage_e[kMaxSlots];
-  float stage_w[kMaxSlots];
   int n_act;
   int last;
   volatile int abort;
@@ -380,9 +390,15 @@ __device__ __forceinline__ void split_bf16x2(float a, float b, uint32_t& head, u
   rest = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-template <bool XBF, int GROUPS, int BLOCKS>  // XBF: token rows are bf16 (else fp32: head + remainder)
+// ROWS = hidden units per stage.  4: the 8 gate / up rows of a stage fill rows 0-7 of the first product's MMAs (rows
+// 8-15 are zeros) and the 4 units half of the second product's k range.  8: a thread also feeds rows gid + 8 (units
+// 4-7) and handles two (unit, token) pairs; both products run at full MMA width, and there are half as many
+// stages, barriers and ldmatrix loads per byte.
+template <bool XBF, int GROUPS, int BLOCKS, int ROWS>  // XBF: token rows are bf16 (else fp32: head + remainder)
 __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm, const Pass& ps, const unsigned char* ring,
                                                  const unsigned char* xs, RingPos& rp, int warp, int lane) {
+  constexpr bool WIDE = ROWS == 8;
+  static_assert(ROWS == 4 || ROWS == 8, "4 or 8 hidden units per stage");
   DeviceState* st = P.st;
   const int NS = P.n_stages, d = P.d, chunks = d >> 3, cl = chunks - 1;
   const int n = ps.ns;
@@ -418,7 +434,9 @@ __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm,
       }
     }
   }
-  const uint32_t row_full = (uint32_t)(gid >> 1) * (uint32_t)P.unit_stride + (uint32_t)(gid & 1) * (uint32_t)(2 * d);
+  // weight row r of a stage (unit r >> 1, gate | up): this thread feeds rows gid and, WIDE, gid + 8
+  const uint32_t row_lo = (uint32_t)(gid >> 1) * (uint32_t)P.unit_stride + (uint32_t)(gid & 1) * (uint32_t)(2 * d);
+  const uint32_t row_hi = row_lo + 4u * (uint32_t)P.unit_stride;
   // (3) output blocks of 16 columns owned by this warp.  ldmatrix: lane i gives the address of row (i & 7) =
   // hidden unit, for columns 8 * (i >> 3) of a pair of blocks; rows and columns that do not exist read zeros.
   const int NB = (d + 15) >> 4;
@@ -433,40 +451,54 @@ __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm,
   for (int bp = 0; bp < BLOCKS; bp += 2) {
     const int col = 16 * (b_lo + bp) + 8 * (lane >> 3);
     lmoff[bp / 2] = (uint32_t)lm_unit * (uint32_t)P.unit_stride + (uint32_t)(4 * d) + (uint32_t)col * 2u;
-    if (col < d && (bp + (lane >> 4)) < b_n && lm_unit < kRows) lmok |= 1u << (bp / 2);
+    if (col < d && (bp + (lane >> 4)) < b_n && lm_unit < ROWS) lmok |= 1u << (bp / 2);
   }
   const uint32_t zero_addr = (uint32_t)__cvta_generic_to_shared(sm.zero16);
   const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(ring);
+  constexpr int kPairs = kRowsWide * 8;  // (unit, token) entries of one gate | up plane of `red`
   float* const red_st = &sm.red[0][gid & 1][(gid >> 1) * 8 + 2 * q][warp];  // + buf * (elements of one buffer)
   const float* const red_ld = &sm.red[0][0][q * 8 + gid][0];
-  constexpr int kRedBuf = 2 * 32 * kWarps;
+  constexpr int kRedBuf = 2 * kPairs * kWarps;
 
   // gate/up partial logits of one stage -> red[stage index & 3]
   auto phase1 = [&](const RingPos& r1, int nrows) {
     const unsigned char* stage = ring + (size_t)r1.slot * P.stage_bytes;
-    const uint32_t rowoff = nrows == kRows ? row_full
-                                           : (uint32_t)min(gid >> 1, nrows - 1) * (uint32_t)P.unit_stride +
-                                                 (uint32_t)(gid & 1) * (uint32_t)(2 * d);
-    const unsigned char* arow = stage + rowoff;
-    uint4 w[GROUPS];
+    // (a ragged last stage: rows of units that do not exist are read from the last unit that does, and never used)
+    const uint32_t off_lo = nrows == ROWS ? row_lo
+                                          : (uint32_t)min(gid >> 1, nrows - 1) * (uint32_t)P.unit_stride +
+                                                (uint32_t)(gid & 1) * (uint32_t)(2 * d);
+    const uint32_t off_hi = nrows == ROWS ? row_hi
+                                          : (uint32_t)min(4 + (gid >> 1), nrows - 1) * (uint32_t)P.unit_stride +
+                                                (uint32_t)(gid & 1) * (uint32_t)(2 * d);
+    const unsigned char* arow = stage + off_lo;
+    const unsigned char* brow = stage + off_hi;
+    uint4 w[GROUPS], w2[WIDE ? GROUPS : 1];
 #pragma unroll
-    for (int gi = 0; gi < GROUPS; ++gi) w[gi] = *reinterpret_cast<const uint4*>(arow + coff[gi]);
+    for (int gi = 0; gi < GROUPS; ++gi) {
+      w[gi] = *reinterpret_cast<const uint4*>(arow + coff[gi]);
+      if (WIDE) w2[WIDE ? gi : 0] = *reinterpret_cast<const uint4*>(brow + coff[gi]);
+    }
     float c[4][4];  // four independent accumulation chains
 #pragma unroll
     for (int j = 0; j < 4; ++j) c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
 #pragma unroll
     for (int gi = 0; gi < GROUPS; ++gi) {
-      mma_16816(c[(2 * gi) & 3], w[gi].x, 0u, w[gi].y, 0u, bh[gi][0], bh[gi][1]);
-      mma_16816(c[(2 * gi + 1) & 3], w[gi].z, 0u, w[gi].w, 0u, bh[gi][2], bh[gi][3]);
+      const uint4 v2 = WIDE ? w2[WIDE ? gi : 0] : make_uint4(0u, 0u, 0u, 0u);
+      mma_16816(c[(2 * gi) & 3], w[gi].x, v2.x, w[gi].y, v2.y, bh[gi][0], bh[gi][1]);
+      mma_16816(c[(2 * gi + 1) & 3], w[gi].z, v2.z, w[gi].w, v2.w, bh[gi][2], bh[gi][3]);
       if (!XBF) {
-        mma_16816(c[(2 * gi + 2) & 3], w[gi].x, 0u, w[gi].y, 0u, bl[XBF ? 0 : gi][0], bl[XBF ? 0 : gi][1]);
-        mma_16816(c[(2 * gi + 3) & 3], w[gi].z, 0u, w[gi].w, 0u, bl[XBF ? 0 : gi][2], bl[XBF ? 0 : gi][3]);
+        mma_16816(c[(2 * gi + 2) & 3], w[gi].x, v2.x, w[gi].y, v2.y, bl[XBF ? 0 : gi][0], bl[XBF ? 0 : gi][1]);
+        mma_16816(c[(2 * gi + 3) & 3], w[gi].z, v2.z, w[gi].w, v2.w, bl[XBF ? 0 : gi][2], bl[XBF ? 0 : gi][3]);
       }
     }
-    // D[row gid][tokens 2q, 2q+1] -> red[buf][gate | up][unit * 8 + token][warp]
+    // D[row gid (and gid + 8)][tokens 2q, 2q+1] -> red[buf][gate | up][unit * 8 + token][warp]
     float* dst = red_st + (r1.n & 3) * kRedBuf;
     dst[0] = (c[0][0] + c[1][0]) + (c[2][0] + c[3][0]);
     dst[kWarps] = (c[0][1] + c[1][1]) + (c[2][1] + c[3][1]);
+    if (WIDE) {  // rows gid + 8: units 4 + (gid >> 1)
+      dst[4 * 8 * kWarps] = (c[0][2] + c[1][2]) + (c[2][2] + c[3][2]);
+      dst[4 * 8 * kWarps + kWarps] = (c[0][3] + c[1][3]) + (c[2][3] + c[3][3]);
+    }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.hbar[r1.slot]);
   };
@@ -480,40 +512,54 @@ __device__ __forceinline__ bool consume_pass_mma(const DenseParams& P, Smem& sm,
       if (lane == 0) set_abort(st, sm, 0x315u);
       return false;
     }
-    phase1(r1, min(kRows, ps.rb - ps.ra));
+    phase1(r1, min(ROWS, ps.rb - ps.ra));
     r1.advance(NS);
   }
-  for (int row0 = ps.ra; row0 < ps.rb; row0 += kRows) {
-    const int nrows = min(kRows, ps.rb - row0);
-    if (row0 + kRows < ps.rb) {
+  for (int row0 = ps.ra; row0 < ps.rb; row0 += ROWS) {
+    const int nrows = min(ROWS, ps.rb - row0);
+    if (row0 + ROWS < ps.rb) {
       if (!mbar_wait(&sm.full[r1.slot], r1.par)) {
         if (lane == 0) set_abort(st, sm, 0x315u);
         return false;
       }
-      phase1(r1, min(kRows, ps.rb - row0 - kRows));
+      phase1(r1, min(ROWS, ps.rb - row0 - ROWS));
       r1.advance(NS);
     }
     if (!mbar_wait_spin(&sm.hbar[rp.slot], rp.par)) {
       if (lane == 0) set_abort(st, sm, 0x316u);
       return false;
     }
-    // ---- (2) lane (token gid, unit q): h
-    float h;
+    // ---- (2) lane (token gid, unit q -- and, WIDE, unit q + 4): h
+    float h, h2 = 0.f;
     {
       const float4* rg = reinterpret_cast<const float4*>(red_ld + (rp.n & 3) * kRedBuf);
-      const float4* ru = rg + 32 * kWarps / 4;
+      const float4* ru = rg + kPairs * kWarps / 4;
       const float4 g0 = rg[0], g1 = rg[1], u0 = ru[0], u1 = ru[1];
       const float g = ((g0.x + g0.y) + (g0.z + g0.w)) + ((g1.x + g1.y) + (g1.z + g1.w));
       const float u = ((u0.x + u0.y) + (u0.z + u0.w)) + ((u1.x + u1.y) + (u1.z + u1.w));
       h = (q < nrows && gid < n) ? g / (1.0f + __expf(-g)) * u : 0.f;  // the gate weight multiplies the pass's sum
+      if (WIDE) {
+        const float4* rg2 = rg + 4 * 8 * kWarps / 4;
+        const float4* ru2 = ru + 4 * 8 * kWarps / 4;
+        const float4 p0 = rg2[0], p1 = rg2[1], v0 = ru2[0], v1 = ru2[1];
+        const float gg = ((p0.x + p0.y) + (p0.z + p0.w)) + ((p1.x + p1.y) + (p1.z + p1.w));
+        const float uu = ((v0.x + v0.y) + (v0.z + v0.w)) + ((v1.x + v1.y) + (v1.z + v1.w));
+        h2 = (q + 4 < nrows && gid < n) ? gg / (1.0f + __expf(-gg)) * uu : 0.f;
+      }
     }
-    // B fragment (k = units 2q, 2q+1 of 8, units 4.. are padding; n = token gid): h rounded to bf16, as the
-    // hidden activations of the tensor-core prefill path are
+    // B fragment (k = units 2q, 2q+1 of 8; n = token gid): h rounded to bf16, as the hidden activations of the
+    // tensor-core prefill path are.  Unit u's value sits in lane (gid, u & 3): as h for u < 4, as h2 above.
     uint32_t hb;
     {
-      const float ha = __shfl_sync(0xffffffffu, h, (lane & ~3) | ((2 * q) & 3));
-      const float hc = __shfl_sync(0xffffffffu, h, (lane & ~3) | ((2 * q + 1) & 3));
-      const __nv_bfloat162 hp = __floats2bfloat162_rn(q < 2 ? ha : 0.f, q < 2 ? hc : 0.f);
+      const int s0 = (lane & ~3) | ((2 * q) & 3), s1 = (lane & ~3) | ((2 * q + 1) & 3);
+      float ha = __shfl_sync(0xffffffffu, h, s0), hc = __shfl_sync(0xffffffffu, h, s1);
+      if (WIDE) {
+        const float ha2 = __shfl_sync(0xffffffffu, h2, s0), hc2 = __shfl_sync(0xffffffffu, h2, s1);
+        if (q >= 2) ha = ha2, hc = hc2;
+      } else if (q >= 2) {
+        ha = hc = 0.f;  // units 4.. are padding
+      }
+      const __nv_bfloat162 hp = __floats2bfloat162_rn(ha, hc);
       hb = *reinterpret_cast<const uint32_t*>(&hp);
     }
     // ---- (3) this warp's output blocks, two per ldmatrix
@@ -743,7 +789,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
   // to the type of x, kept in shared memory as token row 0 and used for the router below.
   const bool from_h = fused1 && P.ex.h_in != nullptr;
   if (from_h) {
-    float* rsum = &sm.red[0][0][0][0];
+    float* rsum = sm.scratch;
     float hv[kRJ];
     float ss = 0.f;
     if (warp < kWarps) {
@@ -903,7 +949,7 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
     // several tokens, E a multiple of 8 (Eq. 2, Eq. 3); every CTA routes all tokens.  A thread owns the input
     // features tid, tid + 256, ...: their router rows are fetched once and serve every token; the tokens go
     // four at a time so that all their loads are in flight together.
-    float* part = &sm.red[0][0][0][0];  // [warp][16 tokens][16 experts]: `red` is not in use before the passes
+    float* part = sm.scratch;  // [warp][16 tokens][16 experts]
     constexpr int XJ = (V == V_MMA_BF16_S || V == V_MMA_F32_S) ? 4 : kXIters;  // features per thread
     constexpr int TC = 32 / XJ;                                                // tokens per round trip
     __syncthreads();  // the barriers the producer thread initialised are waited on below
@@ -1174,13 +1220,14 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
         copy_mask |= 1u << rp.slot;
         rp.advance(NS);
       }
-      for (int row = ps.ra + skip * kRows; P.dyn || row < ps.rb; row += kRows) {
+      const int SR = kAllX ? P.stage_rows : kRows;  // hidden units per stage
+      for (int row = ps.ra + skip * kRows; P.dyn || row < ps.rb; row += SR) {
         int cur = 0;
         if (P.dyn) {
           cur = dyn_next < dyn_stat_end ? dyn_next++ : dyn_base + (int)atomicAdd(&st->stage_ctr[ps.ai], 1u);
           if (cur >= n_st) cur = -1;
         }
-        const int nrows = P.dyn ? (cur < 0 ? 0 : min(kRows, P.f - cur * kRows)) : min(kRows, ps.rb - row);
+        const int nrows = P.dyn ? (cur < 0 ? 0 : min(kRows, P.f - cur * kRows)) : min(SR, ps.rb - row);
         const uint32_t bytes = (uint32_t)nrows * row_bytes;
         if (rp.n >= NS) {
           if (!mbar_wait(&sm.freeb[rp.slot], rp.par ^ 1u)) {
@@ -1257,13 +1304,13 @@ __global__ void __launch_bounds__(kThreads, 1) dense_stream_kernel(const DensePa
       else if (V == V_COLS)
         ok = consume_pass_cols(P, sm, ps, ring, xsb, rp, warp, lane);
       else if (V == V_MMA_BF16_S)
-        ok = consume_pass_mma<true, 4, 8>(P, sm, ps, ring, xsb, rp, warp, lane);
+        ok = consume_pass_mma<true, 4, 8, kRowsWide>(P, sm, ps, ring, xsb, rp, warp, lane);
       else if (V == V_MMA_F32_S)
-        ok = consume_pass_mma<false, 4, 8>(P, sm, ps, ring, xsb, rp, warp, lane);
+        ok = consume_pass_mma<false, 4, 8, kRowsWide>(P, sm, ps, ring, xsb, rp, warp, lane);
       else if (V == V_MMA_BF16_L)
-        ok = consume_pass_mma<true, 8, 16>(P, sm, ps, ring, xsb, rp, warp, lane);
+        ok = consume_pass_mma<true, 8, 16, kRows>(P, sm, ps, ring, xsb, rp, warp, lane);
       else
-        ok = consume_pass_mma<false, 8, 16>(P, sm, ps, ring, xsb, rp, warp, lane);
+        ok = consume_pass_mma<false, 8, 16, kRows>(P, sm, ps, ring, xsb, rp, warp, lane);
       ++pn;
     }
     passes_done = ok ? pn : -1;
@@ -1470,7 +1517,8 @@ int launch_dense_stream(moe_ctx* ctx, int mode, const void* x, int T, const moe_
                      : (xrow + 127) / 128 * 128;
   P.use_mma = T > 1 ? 1 : 0;
   P.unit_stride = 3 * c.d_model * 2 + (P.use_mma ? 16 : 0);  // multiple of 16; the ring base is 128-byte aligned
-  P.stage_bytes = (kRows * P.unit_stride + 127) / 128 * 128;
+  P.stage_rows = (P.use_mma && c.d_model <= 1024) ? kRowsWide : kRows;
+  P.stage_bytes = (P.stage_rows * P.unit_stride + 127) / 128 * 128;
   P.wpart_ok = (!P.use_mma && c.d_model <= 32 * 8 * kT1Iters) ? 1 : 0;
   const size_t fixed = 2 * (size_t)P.xs_bytes + (P.wpart_ok ? (size_t)kWarps * c.d_model * 4 : 0) + kSmemHeaderBytes + 256;
   const long long avail = (long long)ctx->max_smem_optin - (long long)fixed;
