@@ -95,6 +95,14 @@ __global__ void __launch_bounds__(kWdThreads) wd_decode_kernel(const WdParams P)
   const int gw = blockIdx.x * kWdWarps + warp, n_warps = gridDim.x * kWdWarps;
   DeviceState* const st = P.st;
   pdl_launch_dependents();
+  // the router's weights do not depend on any earlier kernel: this thread's rows (first eight experts) are fetched
+  // before the dependency wait, not after the token row behind it
+  uint4 wr0[kWdMaxD / kWdThreads];
+  if ((E & 7) == 0) {
+#pragma unroll
+    for (int q = 0; q < kWdMaxD / kWdThreads; ++q)
+      wr0[q] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + q * kWdThreads, d - 1) * E));
+  }
   pdl_wait();
 
   // ---------------------------------------------------------------- token row, router (every CTA)
@@ -109,7 +117,8 @@ __global__ void __launch_bounds__(kWdThreads) wd_decode_kernel(const WdParams P)
       uint4 wr[kWdMaxD / kWdThreads];  // this thread's router rows, fetched in one round trip
 #pragma unroll
       for (int q = 0; q < kWdMaxD / kWdThreads; ++q)
-        wr[q] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + q * kWdThreads, d - 1) * E + e0));
+        wr[q] = e0 == 0 ? wr0[q]
+                        : __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + q * kWdThreads, d - 1) * E + e0));
 #pragma unroll
       for (int q = 0; q < kWdMaxD / kWdThreads; ++q) {
         const int i = tid + q * kWdThreads;
@@ -383,6 +392,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
     fence_proxy_async_smem();
     sm.abort = 0;
   }
+  uint4 wr0[kWdMaxD / kWdThreads];  // this thread's router rows (first eight experts): constants, fetched before the wait
+  if ((E & 7) == 0 && warp < kWdWarps) {
+#pragma unroll
+    for (int q = 0; q < kWdMaxD / kWdThreads; ++q)
+      wr0[q] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + q * kWdThreads, d - 1) * E));
+  }
   pdl_wait();
 
   // ---------------------------------------------------------------- token row, router (every CTA)
@@ -399,7 +414,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
         uint4 wr[kWdMaxD / kWdThreads];
 #pragma unroll
         for (int q = 0; q < kWdMaxD / kWdThreads; ++q)
-          wr[q] = __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + q * kWdThreads, d - 1) * E + e0));
+          wr[q] = e0 == 0 ? wr0[q]
+                          : __ldg(reinterpret_cast<const uint4*>(P.w_router + (size_t)min(tid + q * kWdThreads, d - 1) * E + e0));
 #pragma unroll
         for (int q = 0; q < kWdMaxD / kWdThreads; ++q) {
           const int i = tid + q * kWdThreads;
