@@ -324,8 +324,9 @@ constexpr int kWsIn = 8;          // 16-byte chunks of the input vector per lane
 struct WsSmem {
   uint64_t full[kWsStages], freeb[kWsStages];
   uint64_t cbar;  // barrier over the consumer warps
-  float x[kWdMaxD];
-  float tg[kWdMaxKR], tu[kWdMaxKR];
+  __align__(16) float x[kWdMaxD];  // (16-byte aligned: the lanes fetch their slices of these vectors as float4)
+  __align__(16) float tg[kWdMaxKR];
+  __align__(16) float tu[kWdMaxKR];
   float rlog[kWdWarps][MOE_MAX_EXPERTS];
   int sel_e[MOE_MAX_TOPK];
   int sel_slot[MOE_MAX_TOPK];
@@ -371,6 +372,16 @@ __device__ __forceinline__ bool ws_meet(DeviceState* st, WsSmem& sm, unsigned& p
     sm.ok = ok;
   }
   return ws_sync(sm, par) && sm.ok != 0;
+}
+
+// eight consecutive fp32 values of a 16-byte aligned vector
+__device__ __forceinline__ void load8f(const float* src, float* dst) {
+  const float4 a = reinterpret_cast<const float4*>(src)[0], b = reinterpret_cast<const float4*>(src)[1];
+  dst[0] = a.x, dst[1] = a.y, dst[2] = a.z, dst[3] = a.w, dst[4] = b.x, dst[5] = b.y, dst[6] = b.z, dst[7] = b.w;
+}
+__device__ __forceinline__ void zero8f(float* dst) {
+#pragma unroll
+  for (int q = 0; q < 8; ++q) dst[q] = 0.f;
 }
 
 __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams P) {
@@ -548,8 +559,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
 #pragma unroll
     for (int j = 0; j < kWsIn; ++j) {
       const int c = lane + 32 * j;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) in[j][q] = c < dc ? sm.x[c * 8 + q] : 0.f;
+      if (c < dc)
+        load8f(sm.x + c * 8, in[j]);
+      else
+        zero8f(in[j]);
     }
     const int N = 2 * r;
     int g0, g1;
@@ -575,10 +588,27 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
     }
   }
   if (!ws_meet(st, sm, cpar)) return;
-  for (int i = tid; i < k * 2 * r; i += kWdThreads) {  // t[a][j][gate|up] -> tg[a][j], tu[a][j]
-    const float v = __ldcg(P.t + i);
-    const int a = i / (2 * r), j2 = i - a * 2 * r;
-    ((j2 & 1) ? sm.tu : sm.tg)[a * r + (j2 >> 1)] = v;
+  {
+    // t[a][j][gate|up] -> tg[a][j], tu[a][j]: four values (two gate / up pairs) per load, all of a thread's loads in
+    // flight together
+    constexpr int kT4 = 2 * kWdMaxKR / 4 / kWdThreads;
+    // (every CTA reads the whole vector in the same order at the same moment: starting each at a different place was
+    // slower -- the L2 serves many requests for one line better than requests spread over all of them)
+    const int n4 = (k * 2 * r) >> 2;
+    float4 v[kT4];
+#pragma unroll
+    for (int u = 0; u < kT4; ++u) {
+      const int l4 = tid + u * kWdThreads, i4 = l4;
+      v[u] = l4 < n4 ? __ldcg(reinterpret_cast<const float4*>(P.t) + i4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kT4; ++u) {
+      const int l4 = tid + u * kWdThreads, i4 = l4;
+      if (l4 < n4) {
+        const int i = 4 * i4, a = i / (2 * r), j = (i - a * 2 * r) >> 1;  // (r is a multiple of 8: a run of 4 stays inside one expert)
+        sm.tg[a * r + j] = v[u].x, sm.tu[a * r + j] = v[u].y, sm.tg[a * r + j + 1] = v[u].z, sm.tu[a * r + j + 1] = v[u].w;
+      }
+    }
   }
   if (!ws_sync(sm, cpar)) return;
 
@@ -595,8 +625,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
         const int c0 = lane + 32 * j;
         up[j] = c0 >= rc;
         const float* src = (up[j] ? sm.tu : sm.tg) + a * r + (c0 - (up[j] ? rc : 0)) * 8;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) in[j][q] = c0 < 2 * rc ? src[q] : 0.f;
+        if (c0 < 2 * rc)
+          load8f(src, in[j]);
+        else
+          zero8f(in[j]);
       }
       for (int r0 = lo; r0 < hi; r0 += kWsRows) {
         const int nr = min(kWsRows, hi - r0);
@@ -620,8 +652,22 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
     }
   }
   if (!ws_meet(st, sm, cpar)) return;
-  for (int i = tid; i < (k * f) >> 2; i += kWdThreads)
-    reinterpret_cast<float4*>(hs)[i] = __ldcg(reinterpret_cast<const float4*>(P.h) + i);
+  {
+    const int n4 = (k * f) >> 2;
+    for (int l0 = tid; l0 < n4; l0 += 8 * kWdThreads) {  // eight loads in flight per thread
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int l = l0 + u * kWdThreads, i = l;
+        v[u] = l < n4 ? __ldcg(reinterpret_cast<const float4*>(P.h) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int l = l0 + u * kWdThreads, i = l;
+        if (l < n4) reinterpret_cast<float4*>(hs)[i] = v[u];
+      }
+    }
+  }
   if (!ws_sync(sm, cpar)) return;
 
   // ---------------------------------------------------------------- v = h dL: rows of f, four partial sums each
@@ -654,9 +700,20 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
     }
   }
   if (!ws_meet(st, sm, cpar)) return;
-  for (int i = tid; i < k * r; i += kWdThreads) {  // v[a][j] = its partial sums, in order
-    const float4 p = __ldcg(reinterpret_cast<const float4*>(P.vpart) + i);
-    sm.tg[i] = ((p.x + p.y) + p.z) + p.w;
+  {
+    constexpr int kV4 = kWdMaxKR / kWdThreads;  // v[a][j] = its partial sums, in order; all of a thread's loads in flight together
+    const int nv = k * r;
+    float4 p[kV4];
+#pragma unroll
+    for (int u = 0; u < kV4; ++u) {
+      const int l = tid + u * kWdThreads, i = l;
+      p[u] = l < nv ? __ldcg(reinterpret_cast<const float4*>(P.vpart) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kV4; ++u) {
+      const int l = tid + u * kWdThreads, i = l;
+      if (l < nv) sm.tg[i] = ((p[u].x + p[u].y) + p[u].z) + p[u].w;
+    }
   }
   if (!ws_sync(sm, cpar)) return;
 
@@ -670,10 +727,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) wd_stream_kernel(const WdParams
       const int a = min(q / rc, k - 1), c = q - a * rc;
       wa[j] = q < k * rc ? sm.sel_w[a] : 0.f;
       off[j] = q < k * rc ? (a * kWsRows * r * 2 + c * 16) : 0;
-#pragma unroll
-      for (int v = 0; v < 8; ++v) in[j][v] = q < k * rc ? sm.tg[q * 8 + v] : 0.f;
+      if (q < k * rc)
+        load8f(sm.tg + q * 8, in[j]);
+      else
+        zero8f(in[j]);
     }
-    const bool good = ld_acquire(&st->status) == 0u;
+    const bool good = ld_relaxed(&st->status) == 0u;  // (ordered behind the meeting's acquire; an acquire of its own would hold the rows back)
     int g0, g1;
     ws_share(P, 3, g0, g1);
     for (int r0 = g0; r0 < g1; r0 += kWsRows) {
