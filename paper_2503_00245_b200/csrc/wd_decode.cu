@@ -44,8 +44,9 @@ struct WdParams {
 };
 
 struct WdSmem {
-  float x[kWdMaxD];
-  float tg[kWdMaxKR], tu[kWdMaxKR];  // t de-interleaved; later v in tg
+  __align__(16) float x[kWdMaxD];   // (16-byte aligned: read as float4)
+  __align__(16) float tg[kWdMaxKR];  // t de-interleaved; later v in tg
+  __align__(16) float tu[kWdMaxKR];
   float rlog[kWdWarps][MOE_MAX_EXPERTS];
   int sel_e[MOE_MAX_TOPK];
   int sel_slot[MOE_MAX_TOPK];
@@ -77,7 +78,17 @@ __device__ __forceinline__ bool meet(DeviceState* st, WdSmem& sm) {
   return sm.ok != 0;
 }
 
-// dot of 8 bf16 weights with 8 fp32 values
+// dot of 8 bf16 weights with 8 fp32 values fetched from a 16-byte aligned place in shared memory as two float4
+__device__ __forceinline__ float dot8s(const uint4& w, const float* v) {
+  const float4 a = reinterpret_cast<const float4*>(v)[0], b = reinterpret_cast<const float4*>(v)[1];
+  float f[8];
+  unpack8(w, f);
+  float acc = f[0] * a.x;
+  acc = fmaf(f[1], a.y, acc), acc = fmaf(f[2], a.z, acc), acc = fmaf(f[3], a.w, acc);
+  acc = fmaf(f[4], b.x, acc), acc = fmaf(f[5], b.y, acc), acc = fmaf(f[6], b.z, acc), acc = fmaf(f[7], b.w, acc);
+  return acc;
+}
+// dot of 8 bf16 weights with 8 fp32 values (registers)
 __device__ __forceinline__ float dot8f(const uint4& w, const float* v) {
   float f[8];
   unpack8(w, f);
@@ -196,7 +207,7 @@ __global__ void __launch_bounds__(kWdThreads) wd_decode_kernel(const WdParams P)
       for (int u = 0; u < 4; ++u) w[u] = __ldg(wrow + min(c0 + 32 * u, dc - 1));
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        if (c0 + 32 * u < dc) acc += dot8f(w[u], sm.x + (c0 + 32 * u) * 8);
+        if (c0 + 32 * u < dc) acc += dot8s(w[u], sm.x + (c0 + 32 * u) * 8);
     }
     acc = warp_sum(acc);
     if (lane == 0) P.t[row] = acc;
@@ -227,7 +238,7 @@ __global__ void __launch_bounds__(kWdThreads) wd_decode_kernel(const WdParams P)
       for (int q = 0; q < 4; ++q) {
         const int u = min(u0 + q * n_warps, k * f - 1);
         const int a = u / f;
-        const float v = dot8f(w[q], (part ? sm.tu : sm.tg) + a * r + cc * 8);
+        const float v = dot8s(w[q], (part ? sm.tu : sm.tg) + a * r + cc * 8);
         if (part) up[q] += v; else g[q] += v;
       }
     }
@@ -287,7 +298,7 @@ __global__ void __launch_bounds__(kWdThreads) wd_decode_kernel(const WdParams P)
     for (int q = lane; q < k * rc; q += 32) {
       const int a = q / rc, c = q - a * rc;
       const uint4 w = __ldg(reinterpret_cast<const uint4*>(P.wd_d + ((size_t)sm.sel_slot[a] * d + i) * r) + c);
-      acc = fmaf(sm.sel_w[a], dot8f(w, sm.tg + a * r + c * 8), acc);
+      acc = fmaf(sm.sel_w[a], dot8s(w, sm.tg + a * r + c * 8), acc);
     }
     acc = warp_sum(acc);
     if (lane == 0 && good) {
