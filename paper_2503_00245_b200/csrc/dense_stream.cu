@@ -9,12 +9,14 @@
 //
 // No second phase, no grid-wide barrier: the CTAs' partial y vectors are summed with 64-bit fixed-point
 // atomics (integer addition is associative, so the sum does not depend on arrival order and repeated
-// calls are bit-identical); the CTA that arrives last converts the sum to the output type and leaves
-// the accumulators zero for the next call.
+// calls are bit-identical).  Who turns the sums into the output: with one token and the whole layer in the
+// launch, the accumulator words count their own arrivals and every CTA finishes a slice of the output by
+// polling its words (see kCntBits); otherwise the last CTAs to arrive at a counter do.  Either way the
+// accumulators are left zero for the next call.
 //
 // (active expert x hidden unit) pairs are split evenly over the CTAs (one per SM).  Inside a CTA:
-//   producer thread   brings stages of 4 hidden units (4 x 3 x d bf16, <= 48 KB) into a ring with one bulk
-//                     asynchronous copy each (TMA without a tensor map), and each pass's token rows of x;
+//   producer thread   brings stages of 4 hidden units (8 with several tokens at d <= 1024; <= 48 KB) into a ring
+//                     with one bulk asynchronous copy each (TMA without a tensor map), and each pass's token rows of x;
 //   8 consumer warps  per stage: (1) one dot product each (4 units x {gate, up}) against the token(s),
 //                     (2) after an mbarrier, each lane owns 8 output columns and adds the 4 units'
 //                     h_c * down_c into register accumulators; at the end of a pass the accumulators go
