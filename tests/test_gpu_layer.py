@@ -236,3 +236,25 @@ def test_streaming_path_writes_y_to_mapped_host_memory(sh, T):
         assert lay.check() == 0
         assert torch.equal(hy, ref.cpu())
     lay.close()
+
+
+@pytest.mark.parametrize("sh", [W.WEARABLE, W.PHONE])
+def test_one_ctx_alternating_token_counts(sh):
+    """One ctx, calls with one token and with several in turn: the two ways of finishing the sums (words that count
+    their arrivals; the arrival counter) share the accumulators, and each must leave them zero for the other.  Every
+    call's output equals that of a fresh ctx given the same rows."""
+    lay, t, _ = U.build(sh, 8, path=STREAM)
+    x8 = t["x"]
+    fresh1, _, _ = U.build(sh, 1, path=STREAM, tensors=t)
+    fresh8, _, _ = U.build(sh, 8, path=STREAM, tensors=t)
+    want8 = fresh8.forward(x8).clone()
+    want1 = [fresh1.forward(x8[i:i + 1]).clone() for i in range(3)]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for i in range(3):
+            assert torch.equal(lay.forward(x8[i:i + 1]), want1[i])
+            assert torch.equal(lay.forward(x8), want8)
+    torch.cuda.synchronize()
+    assert lay.check() == 0 and fresh1.check() == 0 and fresh8.check() == 0
+    for l in (lay, fresh1, fresh8):
+        l.close()
